@@ -1,0 +1,149 @@
+"""fp64 CPU oracle for the GDN speculative verify / accept / commit path.
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT.  Only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import this package.  It shares no code with
+the CUDA library and never imports it.
+
+The arithmetic lives in ``gdn_oracle.c`` (plain C, fp64, the definitions of
+Sections 2.2, 4.2 and 5.1 written out).  This module compiles that file with
+gcc on first use and exposes numpy-in / numpy-out wrappers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gdn_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libgdn_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (gcc, -O2, OpenMP).  Returns the path of the shared object."""
+    with _lock:
+        stale = (not os.path.exists(_LIB_PATH)
+                 or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC))
+        if force or stale:
+            tmp = _LIB_PATH + f".tmp{os.getpid()}"
+            # -ffp-contract=off: no fused multiply-add, every product is rounded
+            # to fp64 before it is added, as written in the source.
+            cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC",
+                   "-shared", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB_PATH)
+        i32, f64, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_decode_step.argtypes = [i32] * 5 + [f64] + [vp] * 7
+        lib.oracle_verify_tree.argtypes = [i32] * 5 + [f64] + [vp] * 9
+        lib.oracle_greedy_accept.argtypes = [i32, i32] + [vp] * 8
+        lib.oracle_commit.argtypes = [i32] * 6 + [vp] * 8
+        _lib = lib
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def decode_step(S, q, k, v, alpha, beta, scale: float = 1.0):
+    """One token per sequence.  S [L,B,H,dv,dk]; q,k uint16 [L,B,H,dk]; v uint16 [L,B,H,dv].
+
+    Returns (S_new float64, o float64 [L,B,H,dv]).  The input is not modified.
+    """
+    S = np.array(S, dtype=np.float64, order="C", copy=True)
+    L, B, H, dv, dk = S.shape
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    alpha, beta = _c(alpha, np.float32), _c(beta, np.float32)
+    assert q.shape == (L, B, H, dk) and k.shape == (L, B, H, dk) and v.shape == (L, B, H, dv)
+    assert alpha.shape == (L, B, H) and beta.shape == (L, B, H)
+    o = np.empty((L, B, H, dv), dtype=np.float64)
+    rc = _load().oracle_decode_step(L, B, H, dk, dv, float(scale), _p(S), _p(q), _p(k), _p(v),
+                                    _p(alpha), _p(beta), _p(o))
+    assert rc == 0
+    return S, o
+
+
+def verify_tree(S0, q, k, v, alpha, beta, node_offsets, parent, scale: float = 1.0):
+    """Outputs of every draft node.  Returns o float64 [L,T,H,dv]."""
+    S0 = _c(S0, np.float64)
+    L, B, H, dv, dk = S0.shape
+    node_offsets, parent = _c(node_offsets, np.int32), _c(parent, np.int32)
+    T = int(node_offsets[B])
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    alpha, beta = _c(alpha, np.float32), _c(beta, np.float32)
+    assert node_offsets.shape == (B + 1,) and parent.shape == (T,)
+    assert q.shape == (L, T, H, dk) and k.shape == (L, T, H, dk) and v.shape == (L, T, H, dv)
+    assert alpha.shape == (L, T, H) and beta.shape == (L, T, H)
+    o = np.zeros((L, T, H, dv), dtype=np.float64)
+    rc = _load().oracle_verify_tree(L, B, H, dk, dv, float(scale), _p(S0), _p(q), _p(k), _p(v),
+                                    _p(alpha), _p(beta), _p(node_offsets), _p(parent), _p(o))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_tree: bad topology (code {rc})")
+    return o
+
+
+def verify_chain(S0, q, k, v, alpha, beta, node_offsets, scale: float = 1.0):
+    """Chain special case: parent[i] = i - 1 inside every sequence."""
+    node_offsets = _c(node_offsets, np.int32)
+    parent = np.concatenate([np.arange(-1, int(n) - 1, dtype=np.int32)
+                             for n in np.diff(node_offsets)] + [np.zeros(0, np.int32)])
+    return verify_tree(S0, q, k, v, alpha, beta, node_offsets, parent, scale)
+
+
+def greedy_accept(node_offsets, parent, draft_tok, target_tok, root_target_tok, max_depth: int):
+    """Returns (path_idx int32 [B,max_depth], path_len int32 [B], next_tok int32 [B])."""
+    node_offsets, parent = _c(node_offsets, np.int32), _c(parent, np.int32)
+    draft_tok, target_tok = _c(draft_tok, np.int32), _c(target_tok, np.int32)
+    root_target_tok = _c(root_target_tok, np.int32)
+    B = node_offsets.shape[0] - 1
+    path_idx = np.empty((B, max_depth), dtype=np.int32)
+    path_len = np.empty((B,), dtype=np.int32)
+    next_tok = np.empty((B,), dtype=np.int32)
+    rc = _load().oracle_greedy_accept(B, int(max_depth), _p(node_offsets), _p(parent),
+                                      _p(draft_tok), _p(target_tok), _p(root_target_tok),
+                                      _p(path_idx), _p(path_len), _p(next_tok))
+    if rc != 0:
+        raise ValueError(f"oracle_greedy_accept: code {rc}")
+    return path_idx, path_len, next_tok
+
+
+def commit(S, k, v, alpha, beta, node_offsets, path_idx, path_len):
+    """Advance the state over the accepted records.  Returns S_new float64 (input untouched)."""
+    S = np.array(S, dtype=np.float64, order="C", copy=True)
+    L, B, H, dv, dk = S.shape
+    node_offsets = _c(node_offsets, np.int32)
+    path_idx, path_len = _c(path_idx, np.int32), _c(path_len, np.int32)
+    T = int(node_offsets[B])
+    max_depth = path_idx.shape[1]
+    k, v = _c(k, np.uint16), _c(v, np.uint16)
+    alpha, beta = _c(alpha, np.float32), _c(beta, np.float32)
+    assert k.shape == (L, T, H, dk) and v.shape == (L, T, H, dv)
+    assert alpha.shape == (L, T, H) and beta.shape == (L, T, H)
+    assert path_idx.shape == (B, max_depth) and path_len.shape == (B,)
+    rc = _load().oracle_commit(L, B, H, dk, dv, max_depth, _p(S), _p(k), _p(v), _p(alpha), _p(beta),
+                               _p(node_offsets), _p(path_idx), _p(path_len))
+    if rc != 0:
+        raise ValueError(f"oracle_commit: bad path (code {rc})")
+    return S

@@ -1,0 +1,439 @@
+"""Pins for the fp64 oracle: what the mathematics and the paper fix, computed by
+routes that share nothing with oracle/gdn_oracle.c.
+
+  * hand-worked scalar cases and closed forms of the gated delta rule
+  * a dense-matrix restatement (transition matrix built explicitly, numpy matmul)
+  * the tree-masked UT/WY factorisation of Section 4.2, solved densely
+  * snapshot propagation over EVERY forest of <= 4 nodes
+  * structural invariants: chain == repeated decode, single-path tree == chain,
+    commit == sequential recurrence, sibling isolation, linearity in (S0, V),
+    row independence, relabelling by another topological order
+  * acceptance: brute force over all root paths, hand cases
+  * byte counts printed by the paper (state, snapshots, factor buffer)
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2607_16673_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------------------
+# independent numpy formulations
+# ---------------------------------------------------------------------------
+def dense_rule(S, k, v, a, b):
+    """S * alpha (I - beta k k^T) + beta v k^T with the d_k x d_k transition matrix formed explicitly."""
+    dk = k.shape[0]
+    return S @ (a * (np.eye(dk) - b * np.outer(k, k))) + b * np.outer(v, k)
+
+
+def snapshot_verify(S0, q, k, v, al, be, parent):
+    """Keep one dense state per node (the 'full-state snapshot' strategy of Section 5.1)."""
+    n = len(parent)
+    states, outs = [None] * n, []
+    for t in range(n):
+        Sp = S0 if parent[t] < 0 else states[parent[t]]
+        states[t] = dense_rule(Sp, k[t], v[t], al[t], be[t])
+        outs.append(states[t] @ q[t])
+    return np.array(outs).reshape(n, S0.shape[0]), states
+
+
+def factorised_verify(S0, q, k, v, al, be, parent):
+    """Tree-masked factorised form (Section 4.2): A_tree = M_tree o (K_b K_a^T),
+    T = (I - A_tree)^-1, O = Qhat S0^T - Attn (W S0^T) + Attn U."""
+    n = len(parent)
+    gamma = np.zeros(n)
+    anc = np.zeros((n, n), dtype=bool)            # strict ancestor mask (M_tree without the diagonal)
+    for t in range(n):
+        p = parent[t]
+        gamma[t] = al[t] * (1.0 if p < 0 else gamma[p])
+        if p >= 0:
+            anc[t] = anc[p]
+            anc[t, p] = True
+    Ka = k / gamma[:, None]
+    Kb = -(be * gamma)[:, None] * k
+    A = np.where(anc, Kb @ Ka.T, 0.0)
+    Tm = np.linalg.inv(np.eye(n) - A)
+    W = Tm @ ((be * gamma)[:, None] * k)
+    Ut = Tm @ (be[:, None] * v)
+    Qh = gamma[:, None] * q
+    Attn = np.where(anc | np.eye(n, dtype=bool), Qh @ Ka.T, 0.0)
+    return Qh @ S0.T - Attn @ (W @ S0.T) + Attn @ Ut
+
+
+def unit_arrays(prob, l=0, b=0, h=0):
+    s, e = int(prob.node_offsets[b]), int(prob.node_offsets[b + 1])
+    f = lambda a: synth.bf16_bits_to_f32(a[l, s:e, h]).astype(np.float64)
+    return (prob.S0[l, b, h].astype(np.float64), f(prob.q), f(prob.k), f(prob.v),
+            prob.alpha[l, s:e, h].astype(np.float64), prob.beta[l, s:e, h].astype(np.float64),
+            prob.parent[s:e])
+
+
+def run_verify(prob, **over):
+    g = lambda name: over.get(name, getattr(prob, name))
+    return oracle.verify_tree(g("S0"), g("q"), g("k"), g("v"), g("alpha"), g("beta"),
+                              g("node_offsets"), g("parent"), prob.scale)
+
+
+def bits(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def one_token(S0, q, k, v, a, b):
+    """Oracle decode of one unit given float arrays (exactly representable in bf16)."""
+    dv, dk = S0.shape
+    S, o = oracle.decode_step(S0[None, None, None], bits(q)[None, None, None], bits(k)[None, None, None],
+                              bits(v)[None, None, None], np.full((1, 1, 1), a, np.float32),
+                              np.full((1, 1, 1), b, np.float32))
+    return S[0, 0, 0], o[0, 0, 0]
+
+
+# ---------------------------------------------------------------------------
+# hand-worked values and closed forms
+# ---------------------------------------------------------------------------
+def test_hand_worked_scalar_cases():
+    """tests/golden/gdn_scalar_cases.txt: 1x1 states worked by hand from the rule."""
+    rows = [r.split() for r in open(os.path.join(GOLDEN, "gdn_scalar_cases.txt"))
+            if r.strip() and not r.startswith("#")]
+    assert len(rows) >= 4
+    for r in rows:
+        S, k, v, a, b, q, S1, o = map(float, r)
+        Sn, on = one_token(np.array([[S]]), [q], [k], [v], a, b)
+        assert Sn[0, 0] == pytest.approx(S1, rel=1e-15, abs=1e-15)
+        assert on[0] == pytest.approx(o, rel=1e-15, abs=1e-15)
+
+
+def test_hand_worked_2x2_case():
+    """S=[[1,2],[3,4]], k=(1,0), v=(5,6), alpha=0.5, beta=0.5, q=(1,1):
+    decayed = [[.5,1],[1.5,2]]; read = (.5,1.5); S' = decayed + .5*(v-read) k^T
+            = [[.5+2.25, 1],[1.5+2.25, 2]] = [[2.75,1],[3.75,2]]; o = (3.75, 5.75)."""
+    Sn, on = one_token(np.array([[1., 2.], [3., 4.]]), [1, 1], [1, 0], [5, 6], 0.5, 0.5)
+    assert np.array_equal(Sn, np.array([[2.75, 1.0], [3.75, 2.0]]))
+    assert np.array_equal(on, np.array([3.75, 5.75]))
+
+
+def test_zero_state_single_token_is_outer_product():
+    rng = np.random.default_rng(1)
+    dk, dv = 16, 8
+    q, k, v, al, be = synth.draw_records(rng, 1, 1, 1, dk, dv)
+    S, o = oracle.decode_step(np.zeros((1, 1, 1, dv, dk)), q, k, v, al, be)
+    kf, vf, qf = (synth.bf16_bits_to_f32(x).astype(np.float64).ravel() for x in (k, v, q))
+    b = float(be.ravel()[0])
+    assert np.allclose(S[0, 0, 0], b * np.outer(vf, kf), rtol=1e-15, atol=0)
+    assert np.allclose(o[0, 0, 0], b * vf * (kf @ qf), rtol=1e-13, atol=1e-15)
+
+
+def test_delta_rule_retrieval_unit_key():
+    """alpha = beta = 1 and |k| = 1  =>  S_1 k = v exactly (the delta rule overwrites the slot)."""
+    rng = np.random.default_rng(2)
+    dk, dv = 64, 32
+    k = rng.choice([-1.0, 1.0], size=dk) / 8.0            # exact in bf16, norm exactly 1
+    v = synth.bf16_bits_to_f32(bits(rng.standard_normal(dv))).astype(np.float64)
+    S0 = rng.standard_normal((dv, dk))
+    S1, _ = one_token(S0, np.zeros(dk), k, v, 1.0, 1.0)
+    assert np.allclose(S1 @ k, v, rtol=0, atol=1e-13)
+    # directions orthogonal to k are untouched
+    w = np.zeros(dk); w[0], w[1] = k[1], -k[0]
+    assert np.allclose(S1 @ w, S0 @ w, rtol=0, atol=1e-13)
+
+
+def test_read_after_write_identity_general():
+    """S_t k_t = alpha (1 - beta |k|^2) S_{t-1} k_t + beta |k|^2 v_t."""
+    rng = np.random.default_rng(3)
+    dk, dv = 32, 16
+    q, k, v, al, be = synth.draw_records(rng, 1, 1, 1, dk, dv)
+    S0 = rng.standard_normal((1, 1, 1, dv, dk))
+    S1, _ = oracle.decode_step(S0, q, k, v, al, be)
+    kf = synth.bf16_bits_to_f32(k).astype(np.float64).ravel()
+    vf = synth.bf16_bits_to_f32(v).astype(np.float64).ravel()
+    a, b, n2 = float(al.ravel()[0]), float(be.ravel()[0]), float(kf @ kf)
+    assert np.allclose(S1[0, 0, 0] @ kf, a * (1 - b * n2) * (S0[0, 0, 0] @ kf) + b * n2 * vf,
+                       rtol=1e-12, atol=1e-13)
+
+
+def test_orthonormal_keys_reduce_to_linear_attention():
+    """alpha = beta = 1, S_0 = 0, orthonormal keys: S_n = sum v_i k_i^T (Eq. 1) and
+    o_n = sum_i v_i (k_i . q_n) -- causal linear attention."""
+    rng = np.random.default_rng(4)
+    dk, dv, n = 16, 8, 6
+    K = np.eye(dk)[:n]
+    V = synth.bf16_bits_to_f32(bits(rng.standard_normal((n, dv)))).astype(np.float64)
+    Q = synth.bf16_bits_to_f32(bits(rng.standard_normal((n, dk)))).astype(np.float64)
+    offs = np.array([0, n], np.int32)
+    ones = np.ones((1, n, 1), np.float32)
+    o = oracle.verify_chain(np.zeros((1, 1, 1, dv, dk)), bits(Q)[None, :, None], bits(K)[None, :, None],
+                            bits(V)[None, :, None], ones, ones, offs)[0, :, 0]
+    expect = np.tril(Q @ K.T) @ V
+    assert np.allclose(o, expect, rtol=0, atol=1e-14)
+    path_idx = np.arange(8, dtype=np.int32)[None]
+    S = oracle.commit(np.zeros((1, 1, 1, dv, dk)), bits(K)[None, :, None], bits(V)[None, :, None], ones, ones,
+                      offs, path_idx, np.array([n], np.int32))
+    assert np.allclose(S[0, 0, 0], V.T @ K, rtol=0, atol=1e-14)
+
+
+def test_beta_zero_is_pure_decay_and_alpha_one_is_identity():
+    prob = synth.make_problem(5, 2, 2, 16, 8, [synth.random_tree_parent(7, 4, 3, np.random.default_rng(5))])
+    zero = np.zeros_like(prob.beta)
+    o = run_verify(prob, beta=zero)
+    S0, q, k, v, al, be, par = unit_arrays(prob, 1, 0, 1)
+    for t in range(len(par)):
+        g = np.prod([al[a] for a in synth.root_path(par, t)])
+        assert np.allclose(o[1, t, 1], g * (S0 @ q[t]), rtol=1e-13, atol=1e-15)
+    one = np.ones_like(prob.alpha)
+    o1 = run_verify(prob, beta=zero, alpha=one)
+    assert np.allclose(o1[1, :, 1], q @ S0.T, rtol=1e-13, atol=1e-15)
+    path = np.full((1, 8), -1, np.int32); path[0, :3] = synth.root_path(par, 6)[:3]
+    n_acc = min(3, len(synth.root_path(par, 6)))
+    Sc = oracle.commit(prob.S0, prob.k, prob.v, one, zero, prob.node_offsets, path, np.array([n_acc], np.int32))
+    assert np.array_equal(Sc, prob.S0.astype(np.float64))
+
+
+# ---------------------------------------------------------------------------
+# independent formulations
+# ---------------------------------------------------------------------------
+def test_decode_matches_dense_matrix_form():
+    rng = np.random.default_rng(6)
+    L, B, H, dk, dv = 2, 3, 2, 24, 12
+    S0 = rng.standard_normal((L, B, H, dv, dk))
+    q, k, v, al, be = synth.draw_records(rng, L, B, H, dk, dv)
+    S1, o = oracle.decode_step(S0, q, k, v, al, be, scale=0.5)
+    f = lambda a: synth.bf16_bits_to_f32(a).astype(np.float64)
+    for l, b, h in itertools.product(range(L), range(B), range(H)):
+        ref = dense_rule(S0[l, b, h], f(k)[l, b, h], f(v)[l, b, h], float(al[l, b, h]), float(be[l, b, h]))
+        assert np.allclose(S1[l, b, h], ref, rtol=1e-12, atol=1e-14)
+        assert np.allclose(o[l, b, h], 0.5 * ref @ f(q)[l, b, h], rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("seed,n,max_depth", [(7, 12, 5), (8, 24, 6), (9, 40, 8)])
+def test_verify_matches_tree_masked_factorisation(seed, n, max_depth):
+    par = synth.random_tree_parent(n, max_depth, 4, np.random.default_rng(seed))
+    prob = synth.make_problem(seed, 1, 2, 32, 16, [par], state_std=0.5)
+    o = run_verify(prob)
+    for h in range(2):
+        S0, q, k, v, al, be, p = unit_arrays(prob, 0, 0, h)
+        ref = factorised_verify(S0, q, k, v, al, be, p)
+        assert np.allclose(o[0, :, h], ref, rtol=1e-9, atol=1e-10)
+
+
+def all_forests(n):
+    return itertools.product(*[range(-1, i) for i in range(n)])
+
+
+def test_brute_force_all_forests_up_to_4_nodes():
+    count = 0
+    for n in range(1, 5):
+        for par in all_forests(n):
+            par = np.array(par, np.int32)
+            prob = synth.make_problem(100 + count, 1, 1, 8, 4, [par], state_std=1.0)
+            o = run_verify(prob)[0, :, 0]
+            S0, q, k, v, al, be, p = unit_arrays(prob)
+            ref, states = snapshot_verify(S0, q, k, v, al, be, p)
+            assert np.allclose(o, ref, rtol=1e-12, atol=1e-13), par
+            # commit along every root path reproduces that node's snapshot
+            for t in range(n):
+                path = synth.root_path(par, t)
+                idx = np.full((1, 8), -1, np.int32); idx[0, :len(path)] = path
+                Sc = oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                                   idx, np.array([len(path)], np.int32))
+                assert np.allclose(Sc[0, 0, 0], states[t], rtol=1e-12, atol=1e-13)
+            count += 1
+    assert count == 1 + 2 + 6 + 24
+
+
+# ---------------------------------------------------------------------------
+# structural invariants
+# ---------------------------------------------------------------------------
+def test_chain_verify_equals_repeated_decode_and_commit():
+    prob = synth.config(1)
+    n = prob.T
+    o = oracle.verify_chain(prob.S0, prob.q, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets)
+    S = prob.S0.astype(np.float64)
+    for t in range(n):
+        S, ot = oracle.decode_step(S, prob.q[:, t:t + 1], prob.k[:, t:t + 1], prob.v[:, t:t + 1],
+                                   prob.alpha[:, t:t + 1], prob.beta[:, t:t + 1])
+        assert np.array_equal(ot[:, 0], o[:, t])          # same arithmetic, same order: bit-identical
+        idx = np.full((1, 8), -1, np.int32); idx[0, :t + 1] = np.arange(t + 1)
+        Sc = oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                           idx, np.array([t + 1], np.int32))
+        assert np.array_equal(Sc, S)
+    # accepted length 0 leaves the state untouched
+    S_same = oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                           np.full((1, 8), -1, np.int32), np.zeros(1, np.int32))
+    assert np.array_equal(S_same, prob.S0.astype(np.float64))
+
+
+def test_single_path_tree_equals_chain():
+    prob = synth.make_problem(11, 2, 2, 16, 16, [synth.chain_parent(6), synth.chain_parent(3)])
+    a = run_verify(prob)
+    b = oracle.verify_chain(prob.S0, prob.q, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets)
+    assert np.array_equal(a, b)
+
+
+def test_root_to_leaf_replay_equals_tree_verify():
+    """Verifying each root path as its own chain (the replay baseline of Section 4.2) gives the same outputs."""
+    par = synth.random_tree_parent(14, 5, 3, np.random.default_rng(12))
+    prob = synth.make_problem(12, 1, 2, 16, 8, [par])
+    o = run_verify(prob)
+    for t in range(14):
+        path = synth.root_path(par, t)
+        sel = np.array(path)
+        oc = oracle.verify_chain(prob.S0, prob.q[:, sel], prob.k[:, sel], prob.v[:, sel], prob.alpha[:, sel],
+                                 prob.beta[:, sel], np.array([0, len(path)], np.int32))
+        assert np.array_equal(oc[:, -1], o[:, t])
+
+
+def test_sibling_isolation():
+    """Changing any factor of node t changes outputs of t and its descendants only (tree mask, Section 4.2)."""
+    rng = np.random.default_rng(13)
+    par = synth.random_tree_parent(16, 5, 3, rng)
+    prob = synth.make_problem(13, 1, 1, 16, 8, [par])
+    base = run_verify(prob)
+    for t in [0, 3, 7, 15]:
+        desc = np.array([t in synth.root_path(par, j) for j in range(16)])
+        for name in ["k", "v", "alpha", "beta"]:
+            arr = getattr(prob, name).copy()
+            if arr.dtype == np.uint16:
+                arr[0, t, 0] = bits(synth.bf16_bits_to_f32(arr[0, t, 0]) * 1.5 + 0.25)
+            else:
+                arr[0, t, 0] = 0.5 * arr[0, t, 0] + 0.1
+            o = run_verify(prob, **{name: arr})
+            changed = np.any(o[0, :, 0] != base[0, :, 0], axis=-1)
+            assert np.array_equal(changed, desc), (t, name)
+        arr = prob.q.copy(); arr[0, t, 0] = bits(synth.bf16_bits_to_f32(arr[0, t, 0]) + 1.0)
+        changed = np.any(run_verify(prob, q=arr)[0, :, 0] != base[0, :, 0], axis=-1)
+        assert np.array_equal(changed, np.arange(16) == t)
+
+
+def test_joint_linearity_in_state_and_values():
+    par = synth.random_tree_parent(10, 4, 3, np.random.default_rng(14))
+    prob = synth.make_problem(14, 1, 2, 16, 8, [par], state_std=1.0)
+    full = run_verify(prob)
+    only_state = run_verify(prob, v=np.zeros_like(prob.v))
+    only_values = run_verify(prob, S0=np.zeros_like(prob.S0))
+    assert np.allclose(full, only_state + only_values, rtol=1e-12, atol=1e-13)
+
+
+def test_row_independence():
+    """Rows of S are independent recurrences (the V-tiling argument, Section 4.1)."""
+    par = synth.random_tree_parent(9, 4, 3, np.random.default_rng(15))
+    prob = synth.make_problem(15, 1, 1, 16, 8, [par], state_std=1.0)
+    perm = np.random.default_rng(15).permutation(8)
+    o = run_verify(prob)
+    op = run_verify(prob, S0=prob.S0[..., perm, :], v=prob.v[..., perm])
+    assert np.array_equal(op, o[..., perm])
+
+
+def test_relabelling_by_another_topological_order():
+    rng = np.random.default_rng(16)
+    par = synth.random_tree_parent(12, 5, 3, rng)
+    prob = synth.make_problem(16, 1, 1, 16, 8, [par])
+    o = run_verify(prob)
+    # DFS preorder is another topological order
+    children = {i: [j for j in range(12) if par[j] == i] for i in range(-1, 12)}
+    order, stack = [], list(reversed(children[-1]))
+    while stack:
+        x = stack.pop(); order.append(x); stack.extend(reversed(children[x]))
+    order = np.array(order); inv = np.empty(12, int); inv[order] = np.arange(12)
+    par2 = np.array([-1 if par[x] < 0 else inv[par[x]] for x in order], np.int32)
+    o2 = run_verify(prob, parent=par2, q=prob.q[:, order], k=prob.k[:, order], v=prob.v[:, order],
+                    alpha=prob.alpha[:, order], beta=prob.beta[:, order])
+    assert np.array_equal(o2, o[:, order])
+
+
+def test_scale_multiplies_outputs():
+    prob = synth.config(1)
+    o1 = run_verify(prob)
+    prob.scale = 0.25
+    assert np.array_equal(run_verify(prob), 0.25 * o1)
+
+
+# ---------------------------------------------------------------------------
+# greedy acceptance
+# ---------------------------------------------------------------------------
+def brute_accept(parent, draft, target, root_target, max_depth):
+    """Enumerate every root path; keep those whose every token equals the prediction made at its parent."""
+    n = len(parent)
+    best = []
+    for t in range(n):
+        path = synth.root_path(parent, t)
+        ok = all(draft[a] == (root_target if parent[a] < 0 else target[parent[a]]) for a in path)
+        if ok and len(path) > len(best):
+            best = path
+    nxt = root_target if not best else target[best[-1]]
+    return best, nxt
+
+
+def accept_one(parent, draft, target, root_target, max_depth=8):
+    parent = np.asarray(parent, np.int32)
+    offs = np.array([0, len(parent)], np.int32)
+    pi, pl, nt = oracle.greedy_accept(offs, parent, np.asarray(draft, np.int32), np.asarray(target, np.int32),
+                                      np.array([root_target], np.int32), max_depth)
+    return list(pi[0, :pl[0]]), int(pl[0]), int(nt[0]), pi[0]
+
+
+def test_accept_hand_cases():
+    # chain 0-1-2, all match
+    assert accept_one([-1, 0, 1], [5, 6, 7], [6, 7, 8], 5)[:3] == ([0, 1, 2], 3, 8)
+    # no match at the root: empty path, next token is the root prediction
+    path, ln, nxt, raw = accept_one([-1, 0, 1], [5, 6, 7], [6, 7, 8], 9)
+    assert (path, ln, nxt) == ([], 0, 9) and np.all(raw == -1)
+    # match stops at an internal node
+    assert accept_one([-1, 0, 1], [5, 6, 7], [6, 1, 8], 5)[:3] == ([0, 1], 2, 1)
+    # the accepted sibling is not the first one; deeper descendant of an unmatched sibling is ignored
+    #      -1 -> 0(tok 3), 1(tok 4);  0 -> 2(tok 9);  1 -> 3(tok 8)
+    assert accept_one([-1, -1, 0, 1], [3, 4, 9, 8], [9, 8, 0, 11], 4)[:3] == ([1, 3], 2, 11)
+    # a descendant that matches its own parent's prediction does not count when the parent is unmatched
+    assert accept_one([-1, 0], [3, 9], [9, 1], 4)[:3] == ([], 0, 4)
+
+
+def test_accept_matches_brute_force_on_random_trees():
+    rng = np.random.default_rng(17)
+    lengths = []
+    for trial in range(200):
+        n = int(rng.integers(1, 20))
+        par = synth.random_tree_parent(n, 8, 4, rng)
+        offs = np.array([0, n], np.int32)
+        draft, target, root = synth.draw_tokens(rng, offs, par, p_match=0.8)
+        path, ln, nxt, _ = accept_one(par, draft, target, int(root[0]))
+        bpath, bnxt = brute_accept(par, draft, target, int(root[0]), 8)
+        assert path == bpath and nxt == bnxt
+        lengths.append(ln)
+    assert max(lengths) >= 3 and min(lengths) == 0
+
+
+def test_accept_batched_offsets():
+    rng = np.random.default_rng(18)
+    parents = synth.ragged_tree_batch(rng, 6, 1, 12, 5)
+    prob = synth.make_problem(18, 1, 1, 8, 8, parents)
+    pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                      prob.root_target_tok, 8)
+    for b in range(6):
+        s, e = prob.node_offsets[b], prob.node_offsets[b + 1]
+        bpath, bnxt = brute_accept(prob.parent[s:e], prob.draft_tok[s:e], prob.target_tok[s:e],
+                                   int(prob.root_target_tok[b]), 8)
+        assert list(pi[b, :pl[b]]) == bpath and nt[b] == bnxt
+
+
+# ---------------------------------------------------------------------------
+# sizes the paper prints (pin the layouts and the record contents)
+# ---------------------------------------------------------------------------
+def test_paper_byte_counts():
+    vals = {}
+    for r in open(os.path.join(GOLDEN, "paper_sizes.txt")):
+        if r.strip() and not r.startswith("#"):
+            key, val = r.split()[:2]
+            vals[key] = float(val)
+    MiB, KiB = 1024 * 1024, 1024
+    state = lambda h, dk, dv: 4 * h * dk * dv
+    assert state(8, 256, 256) == vals["state_MiB_per_layer"] * MiB
+    assert state(32, 128, 128) == vals["state_MiB_per_layer"] * MiB
+    assert 2 * state(8, 256, 256) == vals["round_trip_MiB_per_token"] * MiB
+    assert 8 * state(8, 256, 256) == vals["snapshots_MiB_L8"] * MiB
+    record = lambda h, dk, dv: 4 * h * (dk + dv + 2)          # fp32 {k, v, alpha, beta} per head
+    assert 8 * record(8, 256, 256) == vals["factor_buffer_KiB_L8"] * KiB
+    assert abs(state(8, 256, 256) / record(8, 256, 256) - vals["snapshot_over_factor_ratio"]) < 1.0
