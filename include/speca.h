@@ -1,0 +1,171 @@
+/*
+ * speca.h -- C ABI of libspeca: speculative verification, greedy acceptance and
+ * commit over the recurrent state of a gated-delta-rule (GDN) linear-attention
+ * layer, plus the single-token decode step, as CUDA kernels for NVIDIA B200
+ * (sm_100a).
+ *
+ * Notation.  L layers, B sequences, H heads, d_k key width, d_v value width,
+ * T = node_offsets[B] draft nodes packed over the batch.  A "unit" is one
+ * (layer, sequence, head); units never interact.
+ *
+ * The rule applied by every entry point (GDN layer, Section 2.2; Eq. 1 is its
+ * un-gated, erase-free special case):
+ *
+ *        S' = S * alpha (I - beta k k^T) + beta v k^T          o = scale * S' q
+ *
+ * with S in R^{d_v x d_k}.  Equivalently  S' = alpha S + u k^T  with the
+ * corrected value  u = beta (v - alpha S k).
+ *
+ * Layouts (row-major, last index contiguous), identical in every call:
+ *      S, S0       float   [L][B][H][d_v][d_k]
+ *      q, k        bf16    [L][T][H][d_k]      (16-bit storage, uint16_t here)
+ *      v           bf16    [L][T][H][d_v]
+ *      alpha, beta float   [L][T][H]
+ *      o, u        float   [L][T][H][d_v]
+ *      node_offsets int32  [B+1]   sequence b owns nodes node_offsets[b] .. node_offsets[b+1]-1
+ *      parent, depth, draft_tok, target_tok   int32 [T]
+ * For speca_decode_step there is exactly one token per sequence (T == B).
+ *
+ * Topology contract (parent-pointer array, Section 4.2 and Section 7).  parent[]
+ * holds indices LOCAL to the sequence; -1 means "child of the committed state".
+ * Nodes are in a topological order: parent[i] < i.  Several -1 nodes (a forest)
+ * are legal.  depth[i] = 1 for children of the committed state, else
+ * depth[parent[i]] + 1; it is optional (NULL) and only cross-checked.
+ *
+ * Memory and ownership.  Every pointer except `dims` is a CUDA DEVICE pointer
+ * owned by the caller; `dims` is host memory read during the call only.  No
+ * entry point allocates or frees device memory, synchronises, or keeps state
+ * between calls.  All work is
+ * enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ * and the call returns immediately.  Every tensor base must be 16-byte aligned.
+ * Outputs must not alias inputs; speca_decode_step and speca_commit update S in
+ * place; the verify calls never write S0.
+ *
+ * Errors.  The return value is SPECA_OK or a negative SPECA_ERR_* for anything
+ * the host can see (NULL pointer, unsupported shape, misalignment, bad size,
+ * CUDA launch failure); nothing is launched in that case.  Faults that live in
+ * device memory (bad parent pointer, offsets that decrease, a sequence larger
+ * than dims.max_nodes or deeper than dims.max_depth, an accepted path that is
+ * not a parent chain, a bounded wait that expired) make the kernels skip the
+ * affected sequence -- its outputs and its state stay untouched -- and OR a
+ * SPECA_STATUS_* bit into *status_word, a device int32 the caller zeroes
+ * beforehand and reads back when it wants to know.  No kernel traps.
+ */
+#ifndef SPECA_H
+#define SPECA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECA_VERSION 100
+
+/* return codes */
+#define SPECA_OK                0
+#define SPECA_ERR_NULL         -1   /* a required pointer is NULL                        */
+#define SPECA_ERR_UNSUPPORTED  -2   /* shape outside the supported set (see speca_dims)  */
+#define SPECA_ERR_ALIGN        -3   /* a tensor base is not 16-byte aligned              */
+#define SPECA_ERR_RANGE        -4   /* a count is negative or too large                  */
+#define SPECA_ERR_CUDA         -5   /* the CUDA runtime reported an error at launch      */
+#define SPECA_ERR_WORKSPACE    -6   /* workspace NULL or smaller than required           */
+
+/* bits of *status_word */
+#define SPECA_STATUS_BAD_PARENT   1   /* parent[i] < -1 or parent[i] >= i                          */
+#define SPECA_STATUS_BAD_OFFSETS  2   /* node_offsets not non-decreasing / not ending at T         */
+#define SPECA_STATUS_BAD_PATH     4   /* accepted path is not a chain of parent links from a root  */
+#define SPECA_STATUS_TOO_DEEP     8   /* a node deeper than max_depth / path_len > max_depth       */
+#define SPECA_STATUS_TOO_MANY    16   /* a sequence has more than dims.max_nodes nodes             */
+#define SPECA_STATUS_TIMEOUT     32   /* a bounded device-side wait gave up                        */
+#define SPECA_STATUS_BAD_DEPTH   64   /* depth[] given and inconsistent with parent[]              */
+
+/* verification routes (dims.route) */
+#define SPECA_ROUTE_AUTO        0   /* library picks                                              */
+#define SPECA_ROUTE_SERIAL      1   /* state-resident walk, one rank-1 update per node (Section 4.1) */
+#define SPECA_ROUTE_FACTORIZED  2   /* tree-masked WY form on tensor cores (Section 4.2)           */
+
+typedef struct speca_dims {
+    int32_t n_layers;    /* L >= 1                                                     */
+    int32_t batch;       /* B >= 1                                                     */
+    int32_t heads;       /* H >= 1                                                     */
+    int32_t d_k;         /* 64, 128 or 256                                             */
+    int32_t d_v;         /* multiple of 32, <= 1024                                    */
+    float   scale;       /* o = scale * S q  (1.0f reproduces the paper's minimal form) */
+    int32_t max_depth;   /* longest root path in nodes, 1..16; width of path_idx rows  */
+    int32_t max_nodes;   /* node budget per sequence (Section 6.1), 1..1024            */
+    int32_t route;       /* SPECA_ROUTE_*                                              */
+} speca_dims;
+
+int         speca_version(void);
+const char *speca_strerror(int code);
+
+/* Bytes of caller-provided device scratch the verify calls need for `total_nodes`
+ * packed nodes (topology plan shared by all layers and heads).  Never 0. */
+size_t speca_workspace_bytes(const speca_dims *dims, int32_t total_nodes);
+
+/* Single-token decode step, the autoregressive baseline (Section 2.2: every step
+ * reads the previous state and writes the updated one).  For every unit:
+ * S <- rule(S; k, v, alpha, beta) in place, o = scale * S_new q.  T == B. */
+int speca_decode_step(const speca_dims *dims, float *S,
+                      const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                      const float *alpha, const float *beta, float *o, void *stream);
+
+/* Chain verification (Section 4.1, state-resident serial verification; the
+ * p_j = j-1 special case of Section 7).  Node j of a sequence sees the state after
+ * nodes 0..j of that sequence were applied to S0.  Writes o for every node and,
+ * if u_or_null != NULL, the corrected values u (a WY-style factor record that,
+ * with k and alpha, rebuilds any node's state).  S0 is read once per unit. */
+int speca_verify_chain(const speca_dims *dims, const float *S0,
+                       const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                       const float *alpha, const float *beta,
+                       const int32_t *node_offsets, int32_t total_nodes,
+                       float *o, float *u_or_null,
+                       void *workspace, size_t workspace_bytes,
+                       int32_t *status_word, void *stream);
+
+/* Tree verification (Sections 4.2-4.3).  Node t sees the state obtained by applying
+ * the rule along its own ancestor path root..t starting from S0; siblings never
+ * influence each other and shared prefixes are computed once.  Same outputs as
+ * speca_verify_chain; `depth_or_null` is optional. */
+int speca_verify_tree(const speca_dims *dims, const float *S0,
+                      const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                      const float *alpha, const float *beta,
+                      const int32_t *node_offsets, int32_t total_nodes,
+                      const int32_t *parent, const int32_t *depth_or_null,
+                      float *o, float *u_or_null,
+                      void *workspace, size_t workspace_bytes,
+                      int32_t *status_word, void *stream);
+
+/* Greedy posterior selection (Section 2.1; all end-to-end runs of Section 8 decode
+ * greedily).  With pred(-1) = root_target_tok[b] and pred(i) = target_tok[i], node t is
+ * matched iff draft_tok[t] == pred(parent[t]) and its parent is matched.  Writes the
+ * root path of the deepest matched node (lowest index on ties) to path_idx[b][0..len),
+ * pads the row with -1, path_len[b] = len (0 if the first token already misses), and
+ * next_tok[b] = pred(last accepted node).  Integer-exact. */
+int speca_greedy_accept(int32_t batch, int32_t max_depth,
+                        const int32_t *node_offsets, const int32_t *parent,
+                        const int32_t *draft_tok, const int32_t *target_tok,
+                        const int32_t *root_target_tok,
+                        int32_t *path_idx, int32_t *path_len, int32_t *next_tok,
+                        int32_t *status_word, void *stream);
+
+/* Commit (Section 5.1 factor buffering, Eq. 3; Section 5.2 immediate update): gathers
+ * the factor records (k, v, alpha, beta) on the accepted path path_idx[b][0..path_len[b])
+ * and advances S over them in place, token by token, in fp32.  path_len[b] == 0 leaves
+ * the sequence's state bitwise untouched (it is neither read nor written).  If
+ * parent_or_null is given the path is checked to be a chain of parent links starting at
+ * a child of the committed state; an invalid path skips the sequence. */
+int speca_commit(const speca_dims *dims, float *S,
+                 const uint16_t *k, const uint16_t *v,
+                 const float *alpha, const float *beta,
+                 const int32_t *node_offsets, int32_t total_nodes,
+                 const int32_t *parent_or_null,
+                 const int32_t *path_idx, const int32_t *path_len,
+                 int32_t *status_word, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECA_H */

@@ -1,0 +1,173 @@
+// extern "C" entry points of libspeca: argument validation and kernel dispatch only.
+#include "speca_common.cuh"
+
+using namespace speca;
+
+namespace {
+
+inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+int check_dims(const speca_dims *d)
+{
+    if (d == nullptr) return SPECA_ERR_NULL;
+    if (d->n_layers < 1 || d->batch < 1 || d->heads < 1) return SPECA_ERR_RANGE;
+    if (d->d_k != 64 && d->d_k != 128 && d->d_k != 256) return SPECA_ERR_UNSUPPORTED;
+    if (d->d_v < 32 || d->d_v > 1024 || d->d_v % 32 != 0) return SPECA_ERR_UNSUPPORTED;
+    if (d->max_depth < 1 || d->max_depth > 16) return SPECA_ERR_RANGE;
+    if (d->max_nodes < 1 || d->max_nodes > 1024) return SPECA_ERR_RANGE;
+    if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_FACTORIZED) return SPECA_ERR_UNSUPPORTED;
+    const long long units = 1LL * d->n_layers * d->batch * d->heads;
+    if (units * (d->d_v / 2) > 0x7fffffffLL) return SPECA_ERR_RANGE;       // grid size bound
+    return SPECA_OK;
+}
+
+Params base_params(const speca_dims *d, int32_t total_nodes)
+{
+    Params p{};
+    p.L = d->n_layers; p.B = d->batch; p.H = d->heads; p.T = total_nodes; p.DV = d->d_v;
+    p.scale = d->scale; p.max_depth = d->max_depth; p.max_nodes = d->max_nodes;
+    return p;
+}
+
+inline int cuda_rc(int e) { return e == 0 ? SPECA_OK : SPECA_ERR_CUDA; }
+
+int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, const uint16_t *k,
+                  const uint16_t *v, const float *alpha, const float *beta,
+                  const int32_t *node_offsets, int32_t total_nodes, const int32_t *parent,
+                  const int32_t *depth, bool chain, float *o, float *u, void *workspace,
+                  size_t workspace_bytes, int32_t *status_word, void *stream)
+{
+    int rc = check_dims(dims);
+    if (rc != SPECA_OK) return rc;
+    if (!S0 || !q || !k || !v || !alpha || !beta || !node_offsets || !o || !status_word) return SPECA_ERR_NULL;
+    if (!chain && !parent) return SPECA_ERR_NULL;
+    if (total_nodes < 0) return SPECA_ERR_RANGE;
+    if (1LL * total_nodes > 1LL * dims->batch * dims->max_nodes) return SPECA_ERR_RANGE;
+    if (misaligned(S0) || misaligned(q) || misaligned(k) || misaligned(v) || misaligned(alpha) ||
+        misaligned(beta) || misaligned(o) || (u && misaligned(u)) || misaligned(node_offsets) ||
+        (parent && misaligned(parent)) || (depth && misaligned(depth)))
+        return SPECA_ERR_ALIGN;
+    if (!workspace || misaligned(workspace) ||
+        workspace_bytes < speca::workspace_bytes(dims->batch, total_nodes))
+        return SPECA_ERR_WORKSPACE;
+    if (total_nodes == 0) return SPECA_OK;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Params p = base_params(dims, total_nodes);
+    p.S0 = S0;
+    p.q = reinterpret_cast<const __nv_bfloat16 *>(q);
+    p.k = reinterpret_cast<const __nv_bfloat16 *>(k);
+    p.v = reinterpret_cast<const __nv_bfloat16 *>(v);
+    p.alpha = alpha; p.beta = beta; p.o = o; p.u = u;
+    p.node_offsets = node_offsets; p.parent = parent; p.depth_in = depth;
+    p.status = status_word;
+    p.ws = carve_workspace(workspace, dims->batch, total_nodes);
+    p.n_slots = tree_slots_needed(dims->max_nodes);
+    if (!chain) {
+        rc = cuda_rc(launch_plan(p, st));
+        if (rc != SPECA_OK) return rc;
+    }
+    return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
+}
+
+}  // namespace
+
+extern "C" {
+
+int speca_version(void) { return SPECA_VERSION; }
+
+const char *speca_strerror(int code)
+{
+    switch (code) {
+    case SPECA_OK: return "ok";
+    case SPECA_ERR_NULL: return "a required pointer is NULL";
+    case SPECA_ERR_UNSUPPORTED: return "unsupported shape or route";
+    case SPECA_ERR_ALIGN: return "a tensor base is not 16-byte aligned";
+    case SPECA_ERR_RANGE: return "a count is out of range";
+    case SPECA_ERR_CUDA: return "CUDA launch error";
+    case SPECA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    }
+    return "unknown speca error code";
+}
+
+size_t speca_workspace_bytes(const speca_dims *dims, int32_t total_nodes)
+{
+    if (dims == nullptr || total_nodes < 0 || dims->batch < 1) return 0;
+    return speca::workspace_bytes(dims->batch, total_nodes);
+}
+
+int speca_decode_step(const speca_dims *dims, float *S, const uint16_t *q, const uint16_t *k,
+                      const uint16_t *v, const float *alpha, const float *beta, float *o, void *stream)
+{
+    int rc = check_dims(dims);
+    if (rc != SPECA_OK) return rc;
+    if (!S || !q || !k || !v || !alpha || !beta || !o) return SPECA_ERR_NULL;
+    if (misaligned(S) || misaligned(q) || misaligned(k) || misaligned(v) || misaligned(alpha) ||
+        misaligned(beta) || misaligned(o))
+        return SPECA_ERR_ALIGN;
+    Params p = base_params(dims, dims->batch);
+    p.S = S;
+    p.q = reinterpret_cast<const __nv_bfloat16 *>(q);
+    p.k = reinterpret_cast<const __nv_bfloat16 *>(k);
+    p.v = reinterpret_cast<const __nv_bfloat16 *>(v);
+    p.alpha = alpha; p.beta = beta; p.o = o;
+    return cuda_rc(launch_decode(p, dims->d_k, static_cast<cudaStream_t>(stream)));
+}
+
+int speca_verify_chain(const speca_dims *dims, const float *S0, const uint16_t *q, const uint16_t *k,
+                       const uint16_t *v, const float *alpha, const float *beta,
+                       const int32_t *node_offsets, int32_t total_nodes, float *o, float *u_or_null,
+                       void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream)
+{
+    return verify_common(dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, nullptr, nullptr, true,
+                         o, u_or_null, workspace, workspace_bytes, status_word, stream);
+}
+
+int speca_verify_tree(const speca_dims *dims, const float *S0, const uint16_t *q, const uint16_t *k,
+                      const uint16_t *v, const float *alpha, const float *beta,
+                      const int32_t *node_offsets, int32_t total_nodes, const int32_t *parent,
+                      const int32_t *depth_or_null, float *o, float *u_or_null, void *workspace,
+                      size_t workspace_bytes, int32_t *status_word, void *stream)
+{
+    return verify_common(dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, parent, depth_or_null,
+                         false, o, u_or_null, workspace, workspace_bytes, status_word, stream);
+}
+
+int speca_greedy_accept(int32_t batch, int32_t max_depth, const int32_t *node_offsets,
+                        const int32_t *parent, const int32_t *draft_tok, const int32_t *target_tok,
+                        const int32_t *root_target_tok, int32_t *path_idx, int32_t *path_len,
+                        int32_t *next_tok, int32_t *status_word, void *stream)
+{
+    if (!node_offsets || !parent || !draft_tok || !target_tok || !root_target_tok || !path_idx || !path_len ||
+        !next_tok || !status_word)
+        return SPECA_ERR_NULL;
+    if (batch < 1 || max_depth < 1 || max_depth > 16) return SPECA_ERR_RANGE;
+    return cuda_rc(launch_accept(batch, max_depth, node_offsets, parent, draft_tok, target_tok,
+                                 root_target_tok, path_idx, path_len, next_tok, status_word,
+                                 static_cast<cudaStream_t>(stream)));
+}
+
+int speca_commit(const speca_dims *dims, float *S, const uint16_t *k, const uint16_t *v,
+                 const float *alpha, const float *beta, const int32_t *node_offsets, int32_t total_nodes,
+                 const int32_t *parent_or_null, const int32_t *path_idx, const int32_t *path_len,
+                 int32_t *status_word, void *stream)
+{
+    int rc = check_dims(dims);
+    if (rc != SPECA_OK) return rc;
+    if (!S || !k || !v || !alpha || !beta || !node_offsets || !path_idx || !path_len || !status_word)
+        return SPECA_ERR_NULL;
+    if (total_nodes < 0) return SPECA_ERR_RANGE;
+    if (misaligned(S) || misaligned(k) || misaligned(v) || misaligned(alpha) || misaligned(beta))
+        return SPECA_ERR_ALIGN;
+    if (total_nodes == 0) return SPECA_OK;
+    Params p = base_params(dims, total_nodes);
+    p.S = S;
+    p.k = reinterpret_cast<const __nv_bfloat16 *>(k);
+    p.v = reinterpret_cast<const __nv_bfloat16 *>(v);
+    p.alpha = alpha; p.beta = beta;
+    p.node_offsets = node_offsets; p.parent = parent_or_null;
+    p.path_idx = path_idx; p.path_len = path_len; p.status = status_word;
+    return cuda_rc(launch_commit(p, dims->d_k, static_cast<cudaStream_t>(stream)));
+}
+
+}  // extern "C"

@@ -1,0 +1,193 @@
+// Integer kernels: topology validation + walk schedule ("plan"), and greedy acceptance.
+//
+// The plan is computed once per verify call and shared by every layer, head and
+// value tile of a sequence.  It turns the parent-pointer array (Section 4.2) into a
+// depth-first processing order in which, at every node, children are visited in
+// ascending order of subtree size.  This is the heavy-path idea of the
+// chain-decomposed schedule (Section 4.3) used as a traversal order: the state of a
+// branching node is parked on chip only while its lighter subtrees are walked and is
+// released when its heaviest child starts, so a handful of slots suffice and no
+// boundary state ever goes to HBM.
+#include "speca_common.cuh"
+
+namespace speca {
+
+namespace {
+
+constexpr int kPlanThreads = 128;
+
+// One CTA per sequence.  Dynamic smem: 5 int32 arrays of max_nodes (+1).
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict__ parent,
+            const int32_t *__restrict__ depth_in, int32_t B, int32_t T, int32_t max_depth,
+            int32_t max_nodes, int32_t n_slots, Workspace ws, int32_t *status)
+{
+    extern __shared__ int32_t sm[];
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    __shared__ int32_t s_flag;
+
+    if (b == 0 && tid < 64) ws.ctrl[tid] = 0;          // reset the work-queue counters
+    const int base = node_offsets[b];
+    const int n = node_offsets[b + 1] - base;
+    int fault = 0;
+    if (base < 0 || n < 0 || base + n > T || (b == B - 1 && base + n != T) || (b == 0 && base != 0))
+        fault = SPECA_STATUS_BAD_OFFSETS;
+    else if (n > max_nodes)
+        fault = SPECA_STATUS_TOO_MANY;
+    if (fault) {
+        if (tid == 0) { atomicOr(status, fault); ws.seq_n[b] = -1; }
+        return;
+    }
+    int32_t *par = sm;                       // [n]
+    int32_t *size = par + max_nodes;         // [n]   subtree size
+    int32_t *bef = size + max_nodes;         // [n]   total size of siblings visited before this node
+    int32_t *nlc = bef + max_nodes;          // [n+1] children with children, index shifted by one (slot 0 = committed state)
+    int32_t *ldf = nlc + max_nodes + 1;      // [n]   1 if an earlier sibling has children (register state lost)
+
+    if (tid == 0) s_flag = 0;
+    for (int i = tid; i < n; i += kPlanThreads) { size[i] = 0; nlc[i + 1] = 0; }
+    if (tid == 0) nlc[0] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += kPlanThreads) {
+        int p = parent[base + i];
+        par[i] = p;
+        if (p < -1 || p >= i) atomicOr(&s_flag, SPECA_STATUS_BAD_PARENT);
+    }
+    __syncthreads();
+    if (s_flag) {
+        if (tid == 0) { atomicOr(status, s_flag); ws.seq_n[b] = -1; }
+        return;
+    }
+    // depth and subtree sizes: every node adds itself to all nodes on its root path
+    for (int i = tid; i < n; i += kPlanThreads) {
+        int d = 0;
+        for (int a = i; a >= 0; a = par[a]) { atomicAdd(&size[a], 1); ++d; }
+        ws.depth[base + i] = d;
+        if (d > max_depth) atomicOr(&s_flag, SPECA_STATUS_TOO_DEEP);
+        if (depth_in != nullptr && depth_in[base + i] != d) atomicOr(&s_flag, SPECA_STATUS_BAD_DEPTH);
+    }
+    __syncthreads();
+    if (s_flag) {
+        if (tid == 0) { atomicOr(status, s_flag); ws.seq_n[b] = -1; }
+        return;
+    }
+    for (int i = tid; i < n; i += kPlanThreads) {
+        const int p = par[i], sz = size[i];
+        if (sz > 1) atomicAdd(&nlc[p + 1], 1);
+        int before = 0, lost = 0;
+        for (int s = 0; s < n; ++s) {
+            if (s == i || par[s] != p) continue;
+            const int ss = size[s];
+            if (ss < sz || (ss == sz && s < i)) { before += ss; lost |= (ss > 1); }
+        }
+        bef[i] = before;
+        ldf[i] = lost;
+    }
+    __syncthreads();
+    for (int i = tid; i < n; i += kPlanThreads) {
+        int pos = -1, slot = 0, first = 0;
+        for (int c = i; c >= 0; c = par[c]) {
+            pos += 1 + bef[c];
+            const int a = par[c];
+            if (a >= 0 && nlc[a + 1] >= 2 && bef[c] + size[c] != size[a] - 1) {
+                ++slot;                                   // a's parked state is live while we are below c
+                if (c == i) first = 1;
+            }
+        }
+        const int leaf = (size[i] == 1);
+        int entry = i;
+        if (ldf[i]) {
+            const int p = par[i];
+            entry |= (p < 0 ? kLoadFromS0 : 1 + (slot - first)) << kPlanLoadShift;
+        }
+        if (!leaf && nlc[i + 1] >= 2) {
+            entry |= (1 + slot) << kPlanSaveShift;
+            if (1 + slot > n_slots) atomicOr(&s_flag, SPECA_STATUS_TOO_MANY);
+        }
+        if (leaf) entry |= kPlanLeafBit;
+        ws.plan[base + pos] = entry;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (s_flag) { atomicOr(status, s_flag); ws.seq_n[b] = -1; }
+        else ws.seq_n[b] = n;
+    }
+}
+
+// One warp per sequence.  Each lane takes nodes t = lane, lane+32, ... and walks t's
+// root path checking every token against the prediction made at its parent.
+__global__ void __launch_bounds__(128)
+accept_kernel(int32_t B, int32_t max_depth, const int32_t *__restrict__ node_offsets,
+              const int32_t *__restrict__ parent, const int32_t *__restrict__ draft_tok,
+              const int32_t *__restrict__ target_tok, const int32_t *__restrict__ root_target_tok,
+              int32_t *__restrict__ path_idx, int32_t *__restrict__ path_len,
+              int32_t *__restrict__ next_tok, int32_t *status)
+{
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const int base = node_offsets[b];
+    const int n = node_offsets[b + 1] - base;
+    const int root_pred = root_target_tok[b];
+    int fault = 0;
+    if (base < 0 || n < 0) fault = SPECA_STATUS_BAD_OFFSETS;
+    // best = (depth << 16) | (0xffff - index): max picks the deepest, then the lowest index
+    int best = -1;
+    if (!fault) {
+        for (int t = lane; t < n; t += 32) {
+            int d = 0, ok = 1;
+            for (int a = t; a >= 0;) {
+                const int p = parent[base + a];
+                if (p < -1 || p >= a) { fault |= SPECA_STATUS_BAD_PARENT; ok = 0; break; }
+                const int pred = (p < 0) ? root_pred : target_tok[base + p];
+                if (draft_tok[base + a] != pred) { ok = 0; break; }
+                if (++d > max_depth) { fault |= SPECA_STATUS_TOO_DEEP; ok = 0; break; }
+                a = p;
+            }
+            if (ok && t <= 0xffff) best = max(best, (d << 16) | (0xffff - t));
+        }
+    }
+    if (n > 0x10000) fault |= SPECA_STATUS_TOO_MANY;
+    for (int off = 16; off; off >>= 1) {
+        best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+        fault |= __shfl_xor_sync(0xffffffffu, fault, off);
+    }
+    if (lane != 0) return;
+    if (fault) {                       // skip the sequence: nothing accepted
+        atomicOr(status, fault);
+        best = -1;
+    }
+    const int len = best < 0 ? 0 : (best >> 16);
+    int node = best < 0 ? -1 : 0xffff - (best & 0xffff);
+    path_len[b] = len;
+    next_tok[b] = (node < 0) ? root_pred : target_tok[base + node];
+    for (int d = max_depth - 1; d >= 0; --d) {
+        if (d < len) { path_idx[b * max_depth + d] = node; node = parent[base + node]; }
+        else path_idx[b * max_depth + d] = -1;
+    }
+}
+
+}  // namespace
+
+int launch_plan(const Params &p, cudaStream_t st)
+{
+    const size_t smem = size_t(5 * p.max_nodes + 1) * sizeof(int32_t);
+    plan_kernel<<<p.B, kPlanThreads, smem, st>>>(p.node_offsets, p.parent, p.depth_in, p.B, p.T,
+                                                  p.max_depth, p.max_nodes, p.n_slots, p.ws, p.status);
+    return int(cudaGetLastError());
+}
+
+int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
+                  const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
+                  int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,
+                  cudaStream_t st)
+{
+    const int warps = 4;
+    accept_kernel<<<(B + warps - 1) / warps, warps * 32, 0, st>>>(
+        B, max_depth, node_offsets, parent, draft_tok, target_tok, root_target_tok, path_idx, path_len,
+        next_tok, status);
+    return int(cudaGetLastError());
+}
+
+}  // namespace speca

@@ -1,0 +1,368 @@
+// State-resident serial kernels: single-token decode, serial chain / tree verification
+// and commit.  All three keep a value-tile of the fp32 state in registers with the
+// full key dimension inside the CTA (V-dimension tiling, Section 4.1), so a row's dot
+// products with k and q never leave a sub-warp and there is no cross-block reduction.
+//
+// Thread mapping.  A row of d_k floats is spread over G = d_k/16 adjacent lanes, each
+// holding 16 floats as four float4 taken at stride G (so a sub-warp reads a row with
+// fully coalesced 128-bit loads).  One warp covers 32/G rows per "row set" and RS row
+// sets; k and q are converted from bf16 once per node per lane.  The two row dot
+// products S_p k and S_p q are taken in ONE pass over the registers, then
+//        u = beta (v - alpha S_p k),   o = scale (alpha S_p q + u (k.q)),   S = alpha S_p + u k^T
+// which is the rule of Section 2.2 with o read from the updated state.  Leaves of a
+// draft tree need no state update at all.
+#include "speca_common.cuh"
+
+namespace speca {
+
+namespace {
+
+template <int DK> struct Map {
+    static constexpr int G = DK / 16;          // lanes per row
+    static constexpr int RPS = 32 / G;         // rows per warp per row set
+};
+
+template <int G> __device__ __forceinline__ float group_sum(float x)
+{
+#pragma unroll
+    for (int off = G / 2; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+
+// 16 of a row's d_k values for this lane, from a bf16 vector in global memory.
+template <int G> __device__ __forceinline__ void load_vec(const __nv_bfloat16 *p, int g, float (&x)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(p) + g + G * c);
+        x[4 * c + 0] = __uint_as_float(raw.x << 16);
+        x[4 * c + 1] = __uint_as_float(raw.x & 0xffff0000u);
+        x[4 * c + 2] = __uint_as_float(raw.y << 16);
+        x[4 * c + 3] = __uint_as_float(raw.y & 0xffff0000u);
+    }
+}
+
+template <int G> __device__ __forceinline__ void load_row(const float *row, int g, float (&s)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const float4 t = *(reinterpret_cast<const float4 *>(row) + g + G * c);
+        s[4 * c + 0] = t.x; s[4 * c + 1] = t.y; s[4 * c + 2] = t.z; s[4 * c + 3] = t.w;
+    }
+}
+
+template <int G> __device__ __forceinline__ void store_row(float *row, int g, const float (&s)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        *(reinterpret_cast<float4 *>(row) + g + G * c) =
+            make_float4(s[4 * c + 0], s[4 * c + 1], s[4 * c + 2], s[4 * c + 3]);
+}
+
+__device__ __forceinline__ float dot16(const float (&a)[16], const float (&b)[16])
+{
+    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) { acc0 = fmaf(a[i], b[i], acc0); acc1 = fmaf(a[i + 1], b[i + 1], acc1); }
+    return acc0 + acc1;
+}
+
+__device__ __forceinline__ float bf16_to_float(const __nv_bfloat16 *p)
+{
+    return __uint_as_float(uint32_t(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+}
+
+// ---------------------------------------------------------------------------
+// decode step: S in place, one token per sequence
+// ---------------------------------------------------------------------------
+template <int DK, int RS, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+decode_kernel(Params p)
+{
+    constexpr int G = Map<DK>::G, RPS = Map<DK>::RPS, ROWS = WARPS * RS * RPS;
+    const int tiles = p.DV / ROWS;
+    const long unit = blockIdx.x / tiles;                       // (l*B + b)*H + h == record index (T == B)
+    const int row0 = (blockIdx.x % tiles) * ROWS + (threadIdx.x >> 5) * RS * RPS;
+    const int lane = threadIdx.x & 31, g = lane % G, sub = lane / G;
+
+    float *Su = p.S + unit * p.DV * DK;
+    float s[RS][16];
+#pragma unroll
+    for (int r = 0; r < RS; ++r) load_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
+    float kx[16], qx[16];
+    load_vec<G>(p.k + unit * DK, g, kx);
+    load_vec<G>(p.q + unit * DK, g, qx);
+    const float alpha = __ldg(p.alpha + unit), beta = __ldg(p.beta + unit);
+    const float kq = group_sum<G>(dot16(kx, qx));
+#pragma unroll
+    for (int r = 0; r < RS; ++r) {
+        const int row = row0 + r * RPS + sub;
+        const float sk = group_sum<G>(dot16(s[r], kx));
+        const float sq = group_sum<G>(dot16(s[r], qx));
+        const float vv = bf16_to_float(p.v + unit * p.DV + row);
+        const float u = beta * (vv - alpha * sk);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
+        store_row<G>(Su + long(row) * DK, g, s[r]);
+        if (g == 0) p.o[unit * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// serial verification (chain: nodes in index order; tree: plan order with slots)
+// ---------------------------------------------------------------------------
+template <int DK, int RS, int WARPS, bool CHAIN>
+__global__ void __launch_bounds__(WARPS * 32)
+verify_serial_kernel(Params p)
+{
+    constexpr int G = Map<DK>::G, RPS = Map<DK>::RPS, ROWS = WARPS * RS * RPS;
+    extern __shared__ float4 slot_mem[];                         // [n_slots][ROWS][DK] floats
+    const int tiles = p.DV / ROWS;
+    const long unit = blockIdx.x / tiles;
+    const int h = int(unit % p.H), b = int((unit / p.H) % p.B), l = int(unit / (long(p.H) * p.B));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane % G, sub = lane / G;
+    const int row0 = (blockIdx.x % tiles) * ROWS + warp * RS * RPS;
+
+    const int base = __ldg(p.node_offsets + b);
+    int n;
+    if (CHAIN) {
+        n = __ldg(p.node_offsets + b + 1) - base;
+        int fault = 0;
+        if (base < 0 || n < 0 || base + n > p.T) fault = SPECA_STATUS_BAD_OFFSETS;
+        else if (n > p.max_nodes) fault = SPECA_STATUS_TOO_MANY;
+        if (fault) {
+            if (threadIdx.x == 0 && blockIdx.x % tiles == 0 && h == 0 && l == 0) atomicOr(p.status, fault);
+            return;
+        }
+    } else {
+        n = p.ws.seq_n[b];
+    }
+    if (n <= 0) return;
+
+    const float *S0u = p.S0 + unit * p.DV * DK;
+    float s[RS][16];
+#pragma unroll
+    for (int r = 0; r < RS; ++r) load_row<G>(S0u + long(row0 + r * RPS + sub) * DK, g, s[r]);
+    float *my_slot = reinterpret_cast<float *>(slot_mem) + size_t(warp) * RS * RPS * DK;
+    const size_t slot_stride = size_t(ROWS) * DK;
+
+    for (int j = 0; j < n; ++j) {
+        int t = j, load = 0, save = 0;
+        bool leaf = (j == n - 1);
+        if (!CHAIN) {
+            const int e = __ldg(p.ws.plan + base + j);
+            t = e & 0xffff;
+            load = (e >> kPlanLoadShift) & 15;
+            save = (e >> kPlanSaveShift) & 15;
+            leaf = (e & kPlanLeafBit) != 0;
+            if (load == kLoadFromS0) {
+#pragma unroll
+                for (int r = 0; r < RS; ++r) load_row<G>(S0u + long(row0 + r * RPS + sub) * DK, g, s[r]);
+            } else if (load) {
+                const float *src = my_slot + slot_stride * (load - 1);
+#pragma unroll
+                for (int r = 0; r < RS; ++r) load_row<G>(src + (r * RPS + sub) * DK, g, s[r]);
+            }
+        }
+        const long rec = (long(l) * p.T + base + t) * p.H + h;
+        float kx[16], qx[16];
+        load_vec<G>(p.k + rec * DK, g, kx);
+        load_vec<G>(p.q + rec * DK, g, qx);
+        const float alpha = __ldg(p.alpha + rec), beta = __ldg(p.beta + rec);
+        const float kq = group_sum<G>(dot16(kx, qx));
+#pragma unroll
+        for (int r = 0; r < RS; ++r) {
+            const int row = row0 + r * RPS + sub;
+            const float sk = group_sum<G>(dot16(s[r], kx));
+            const float sq = group_sum<G>(dot16(s[r], qx));
+            const float vv = bf16_to_float(p.v + rec * p.DV + row);
+            const float u = beta * (vv - alpha * sk);
+            if (!leaf) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
+            }
+            if (g == 0) {
+                p.o[rec * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
+                if (p.u != nullptr) p.u[rec * p.DV + row] = u;
+            }
+        }
+        if (!CHAIN && save) {
+            float *dst = my_slot + slot_stride * (save - 1);
+#pragma unroll
+            for (int r = 0; r < RS; ++r) store_row<G>(dst + (r * RPS + sub) * DK, g, s[r]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// commit: advance S in place over the accepted factor records
+// ---------------------------------------------------------------------------
+template <int DK, int RS, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+commit_kernel(Params p)
+{
+    constexpr int G = Map<DK>::G, RPS = Map<DK>::RPS, ROWS = WARPS * RS * RPS;
+    const int tiles = p.DV / ROWS;
+    const long unit = blockIdx.x / tiles;
+    const int h = int(unit % p.H), b = int((unit / p.H) % p.B), l = int(unit / (long(p.H) * p.B));
+    const int lane = threadIdx.x & 31, g = lane % G, sub = lane / G;
+    const int row0 = (blockIdx.x % tiles) * ROWS + (threadIdx.x >> 5) * RS * RPS;
+
+    const int len = __ldg(p.path_len + b);
+    if (len == 0) return;
+    const int base = __ldg(p.node_offsets + b);
+    const int n = __ldg(p.node_offsets + b + 1) - base;
+    // validate the whole path before touching the state (uniform over the CTA)
+    int fault = 0;
+    if (len < 0 || len > p.max_depth) fault = SPECA_STATUS_TOO_DEEP;
+    else if (base < 0 || n < 0 || base + n > p.T) fault = SPECA_STATUS_BAD_OFFSETS;
+    else {
+        int prev = -1;
+        for (int d = 0; d < len; ++d) {
+            const int t = __ldg(p.path_idx + b * p.max_depth + d);
+            if (t < 0 || t >= n) { fault = SPECA_STATUS_BAD_PATH; break; }
+            if (p.parent != nullptr && __ldg(p.parent + base + t) != prev) { fault = SPECA_STATUS_BAD_PATH; break; }
+            prev = t;
+        }
+    }
+    if (fault) {
+        if (threadIdx.x == 0 && blockIdx.x % tiles == 0 && h == 0 && l == 0) atomicOr(p.status, fault);
+        return;
+    }
+
+    float *Su = p.S + unit * p.DV * DK;
+    float s[RS][16];
+#pragma unroll
+    for (int r = 0; r < RS; ++r) load_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
+    for (int d = 0; d < len; ++d) {
+        const int t = __ldg(p.path_idx + b * p.max_depth + d);
+        const long rec = (long(l) * p.T + base + t) * p.H + h;
+        float kx[16];
+        load_vec<G>(p.k + rec * DK, g, kx);
+        const float alpha = __ldg(p.alpha + rec), beta = __ldg(p.beta + rec);
+#pragma unroll
+        for (int r = 0; r < RS; ++r) {
+            const int row = row0 + r * RPS + sub;
+            const float sk = group_sum<G>(dot16(s[r], kx));
+            const float vv = bf16_to_float(p.v + rec * p.DV + row);
+            const float u = beta * (vv - alpha * sk);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < RS; ++r) store_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
+}
+
+// Rows covered by one CTA for a given d_k: the largest of {32,16,8,4,2} rows (RS in
+// {2,1}) that divides d_v is chosen by the launchers below.
+template <int DK, int RS, int WARPS> constexpr int rows_per_cta() { return WARPS * RS * Map<DK>::RPS; }
+
+template <int DK, template <int, int, int> class Launch>
+int pick_tile(const Params &p, cudaStream_t st)
+{
+    // prefer 2 row sets x 4 warps; fall back to smaller tiles when d_v is not a multiple
+    if (p.DV % rows_per_cta<DK, 2, 4>() == 0) return Launch<DK, 2, 4>::run(p, st);
+    if (p.DV % rows_per_cta<DK, 2, 2>() == 0) return Launch<DK, 2, 2>::run(p, st);
+    if (p.DV % rows_per_cta<DK, 1, 2>() == 0) return Launch<DK, 1, 2>::run(p, st);
+    if (p.DV % rows_per_cta<DK, 1, 1>() == 0) return Launch<DK, 1, 1>::run(p, st);
+    return int(cudaErrorInvalidValue);
+}
+
+inline long n_units(const Params &p) { return long(p.L) * p.B * p.H; }
+
+template <int DK, int RS, int WARPS> struct LaunchDecode {
+    static int run(const Params &p, cudaStream_t st)
+    {
+        const long blocks = n_units(p) * (p.DV / rows_per_cta<DK, RS, WARPS>());
+        decode_kernel<DK, RS, WARPS><<<unsigned(blocks), WARPS * 32, 0, st>>>(p);
+        return int(cudaGetLastError());
+    }
+};
+
+template <int DK, int RS, int WARPS> struct LaunchCommit {
+    static int run(const Params &p, cudaStream_t st)
+    {
+        const long blocks = n_units(p) * (p.DV / rows_per_cta<DK, RS, WARPS>());
+        commit_kernel<DK, RS, WARPS><<<unsigned(blocks), WARPS * 32, 0, st>>>(p);
+        return int(cudaGetLastError());
+    }
+};
+
+template <int DK, int RS, int WARPS> struct LaunchChain {
+    static int run(const Params &p, cudaStream_t st)
+    {
+        const long blocks = n_units(p) * (p.DV / rows_per_cta<DK, RS, WARPS>());
+        verify_serial_kernel<DK, RS, WARPS, true><<<unsigned(blocks), WARPS * 32, 0, st>>>(p);
+        return int(cudaGetLastError());
+    }
+};
+
+template <int DK, int RS, int WARPS> struct LaunchTree {
+    static int run(const Params &p, cudaStream_t st)
+    {
+        constexpr int ROWS = rows_per_cta<DK, RS, WARPS>();
+        const long blocks = n_units(p) * (p.DV / ROWS);
+        const size_t smem = size_t(p.n_slots) * ROWS * DK * sizeof(float);
+        auto kern = verify_serial_kernel<DK, RS, WARPS, false>;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            if (e != cudaSuccess) return int(e);
+        }
+        kern<<<unsigned(blocks), WARPS * 32, smem, st>>>(p);
+        return int(cudaGetLastError());
+    }
+};
+
+// The tree walk parks whole tiles on chip, so it uses a smaller tile (2 warps) to keep
+// several CTAs resident per SM.
+template <int DK>
+int pick_tree_tile(const Params &p, cudaStream_t st)
+{
+    if (p.DV % rows_per_cta<DK, 2, 2>() == 0) return LaunchTree<DK, 2, 2>::run(p, st);
+    if (p.DV % rows_per_cta<DK, 1, 2>() == 0) return LaunchTree<DK, 1, 2>::run(p, st);
+    if (p.DV % rows_per_cta<DK, 1, 1>() == 0) return LaunchTree<DK, 1, 1>::run(p, st);
+    return int(cudaErrorInvalidValue);
+}
+
+}  // namespace
+
+int launch_decode(const Params &p, int d_k, cudaStream_t st)
+{
+    switch (d_k) {
+    case 64: return pick_tile<64, LaunchDecode>(p, st);
+    case 128: return pick_tile<128, LaunchDecode>(p, st);
+    case 256: return pick_tile<256, LaunchDecode>(p, st);
+    }
+    return int(cudaErrorInvalidValue);
+}
+
+int launch_commit(const Params &p, int d_k, cudaStream_t st)
+{
+    switch (d_k) {
+    case 64: return pick_tile<64, LaunchCommit>(p, st);
+    case 128: return pick_tile<128, LaunchCommit>(p, st);
+    case 256: return pick_tile<256, LaunchCommit>(p, st);
+    }
+    return int(cudaErrorInvalidValue);
+}
+
+int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st)
+{
+    if (chain) {
+        switch (d_k) {
+        case 64: return pick_tile<64, LaunchChain>(p, st);
+        case 128: return pick_tile<128, LaunchChain>(p, st);
+        case 256: return pick_tile<256, LaunchChain>(p, st);
+        }
+    } else {
+        switch (d_k) {
+        case 64: return pick_tree_tile<64>(p, st);
+        case 128: return pick_tree_tile<128>(p, st);
+        case 256: return pick_tree_tile<256>(p, st);
+        }
+    }
+    return int(cudaErrorInvalidValue);
+}
+
+}  // namespace speca

@@ -1,0 +1,102 @@
+// Shared declarations of the libspeca translation units (device helpers, launch
+// parameter blocks, workspace layout).  Nothing here is visible at the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/speca.h"
+
+namespace speca {
+
+// ---------------------------------------------------------------------------
+// Workspace layout (device scratch handed in by the caller).
+//   [0, 256)                     control words (work-queue counters)
+//   [256, 256 + 4*Bpad)          seq_n[b]: node count of sequence b, or -1 if the
+//                                sequence failed validation and must be skipped
+//   then 4 int32 arrays of Tpad: plan[], depth[], anc_lo[], anc_hi[] ...
+// Every region starts on a 256-byte boundary.
+// ---------------------------------------------------------------------------
+constexpr size_t kCtrlBytes = 256;
+constexpr int kNodeWords = 16;          // int32 words of scratch reserved per packed node
+
+__host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct Workspace {
+    int32_t *ctrl;      // [64]
+    int32_t *seq_n;     // [B]
+    int32_t *plan;      // [T]   packed schedule entries, in processing order per sequence
+    int32_t *depth;     // [T]   depth computed from parent[]
+    int32_t *anc;       // [T][kMaxDepthWords] reserved for the factorised route
+};
+
+inline size_t workspace_bytes(int32_t batch, int32_t total_nodes)
+{
+    return kCtrlBytes + align256(size_t(batch) * 4) + align256(size_t(total_nodes) * 4) * kNodeWords;
+}
+
+inline Workspace carve_workspace(void *base, int32_t batch, int32_t total_nodes)
+{
+    Workspace w;
+    char *p = static_cast<char *>(base);
+    w.ctrl = reinterpret_cast<int32_t *>(p);
+    p += kCtrlBytes;
+    w.seq_n = reinterpret_cast<int32_t *>(p);
+    p += align256(size_t(batch) * 4);
+    size_t tb = align256(size_t(total_nodes) * 4);
+    w.plan = reinterpret_cast<int32_t *>(p);
+    w.depth = reinterpret_cast<int32_t *>(p + tb);
+    w.anc = reinterpret_cast<int32_t *>(p + 2 * tb);
+    return w;
+}
+
+// Packed schedule entry written by the plan kernel, one per node, in the order
+// the serial tree walk processes the nodes of a sequence.
+//   bits  0..15  node index (local to the sequence)
+//   bits 16..19  load code: 0 = parent state is already in registers,
+//                1..14 = reload from on-chip slot (code-1), 15 = reload S0 from HBM
+//   bits 20..23  save code: 0 = none, 1..14 = store the new state to slot (code-1)
+//   bit  24      leaf: emit o only, leave the register state at the parent's
+constexpr int kPlanLoadShift = 16, kPlanSaveShift = 20, kPlanLeafBit = 1 << 24;
+constexpr int kLoadFromS0 = 15;
+
+// Launch parameter block shared by the kernels.
+struct Params {
+    int32_t L, B, H, T, DV;
+    float scale;
+    int32_t max_depth, max_nodes;
+    float *S;                    // in/out for decode and commit
+    const float *S0;             // read-only for verify
+    const __nv_bfloat16 *q, *k, *v;
+    const float *alpha, *beta;
+    float *o, *u;
+    const int32_t *node_offsets, *parent, *depth_in;
+    const int32_t *path_idx, *path_len;
+    int32_t *status;
+    Workspace ws;
+    int32_t n_slots;             // on-chip state slots available to the tree walk
+};
+
+// Launchers implemented per translation unit; each returns a cudaError_t-compatible int.
+int launch_plan(const Params &p, cudaStream_t st);
+int launch_decode(const Params &p, int d_k, cudaStream_t st);
+int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
+int launch_commit(const Params &p, int d_k, cudaStream_t st);
+int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
+                  const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
+                  int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,
+                  cudaStream_t st);
+
+// Number of on-chip state slots the light-children-first walk can need for a tree of
+// at most n nodes: a node saves its state only if it has two children with
+// children of their own (subtree >= 5 nodes) and every live slot at least halves
+// the remaining subtree.
+inline int tree_slots_needed(int n)
+{
+    int s = 0;
+    while (n >= 5) { ++s; n = (n - 1) / 2; }
+    return s;
+}
+
+}  // namespace speca

@@ -1,0 +1,97 @@
+"""Helpers shared by the GPU parity tests: upload a synthetic problem, call the
+C ABI through the binding, compare with the oracle."""
+import numpy as np
+import torch
+
+from paper_2607_16673_b200 import binding as speca
+from paper_2607_16673_b200 import synth
+
+# Parity bar of the benchmark spec: outputs and committed states within 2e-3 of the
+# fp64 oracle, measured as max |x - r| / (|r| + rms(r)) over one output tensor (a
+# pure element-wise relative error is meaningless where outputs cross zero).
+TOL = 2e-3
+# fp32 kernels (state-resident serial route, decode, commit): every element is a
+# sum of <= d_k + depth products of O(1) terms accumulated in fp32; with d_k = 256
+# and depth 16 a loose bound is 300 * 2^-24 ~ 2e-5 relative to the tensor's scale.
+TOL_FP32 = 2e-5
+
+
+def rel_err(x, r) -> float:
+    x = np.asarray(x, dtype=np.float64)
+    r = np.asarray(r, dtype=np.float64)
+    if r.size == 0:
+        return 0.0
+    rms = float(np.sqrt(np.mean(r * r)))
+    return float(np.max(np.abs(x - r) / (np.abs(r) + rms + 1e-300)))
+
+
+def bf16_dev(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DevProblem:
+    """A synth.Problem resident on the GPU plus output buffers."""
+
+    def __init__(self, prob: synth.Problem, route=speca.ROUTE_AUTO, max_nodes=None, want_u=False,
+                 device="cuda"):
+        self.prob = prob
+        sizes = np.diff(prob.node_offsets)
+        if max_nodes is None:
+            max_nodes = max(1, int(sizes.max()) if sizes.size else 1)
+        self.dims = speca.Dims(prob.L, prob.B, prob.H, prob.d_k, prob.d_v, prob.scale, prob.max_depth,
+                               max_nodes, route)
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+        self.S = t(prob.S0)
+        self.q, self.k, self.v = bf16_dev(prob.q, device), bf16_dev(prob.k, device), bf16_dev(prob.v, device)
+        self.alpha, self.beta = t(prob.alpha), t(prob.beta)
+        self.node_offsets, self.parent, self.depth = t(prob.node_offsets), t(prob.parent), t(prob.depth)
+        self.draft_tok, self.target_tok = t(prob.draft_tok), t(prob.target_tok)
+        self.root_target_tok = t(prob.root_target_tok)
+        T = prob.T
+        self.T = T
+        self.o = torch.full((prob.L, T, prob.H, prob.d_v), float("nan"), device=device)
+        self.u = torch.full((prob.L, T, prob.H, prob.d_v), float("nan"), device=device) if want_u else None
+        self.ws = speca.alloc_workspace(self.dims, T, device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.path_idx = torch.full((prob.B, prob.max_depth), -7, dtype=torch.int32, device=device)
+        self.path_len = torch.full((prob.B,), -7, dtype=torch.int32, device=device)
+        self.next_tok = torch.full((prob.B,), -7, dtype=torch.int32, device=device)
+        if prob.path_idx is not None:
+            self.path_idx.copy_(t(prob.path_idx))
+            self.path_len.copy_(t(prob.path_len))
+
+    def verify_tree(self, with_depth=True):
+        speca.verify_tree(self.dims, self.S, self.q, self.k, self.v, self.alpha, self.beta, self.node_offsets,
+                          self.T, self.parent, self.depth if with_depth else None, self.o, self.u, self.ws,
+                          self.status)
+        return self.o
+
+    def verify_chain(self):
+        speca.verify_chain(self.dims, self.S, self.q, self.k, self.v, self.alpha, self.beta, self.node_offsets,
+                           self.T, self.o, self.u, self.ws, self.status)
+        return self.o
+
+    def accept(self):
+        speca.greedy_accept(self.prob.B, self.prob.max_depth, self.node_offsets, self.parent, self.draft_tok,
+                            self.target_tok, self.root_target_tok, self.path_idx, self.path_len, self.next_tok,
+                            self.status)
+
+    def commit(self, check_parent=True):
+        speca.commit(self.dims, self.S, self.k, self.v, self.alpha, self.beta, self.node_offsets, self.T,
+                     self.parent if check_parent else None, self.path_idx, self.path_len, self.status)
+
+    def status_value(self) -> int:
+        torch.cuda.synchronize()
+        return int(self.status.item())
+
+
+def oracle_verify(prob):
+    import oracle
+    return oracle.verify_tree(prob.S0, prob.q, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                              prob.parent, prob.scale)
+
+
+def oracle_commit(prob, path_idx, path_len, S=None):
+    import oracle
+    return oracle.commit(prob.S0 if S is None else S, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                         path_idx, path_len)

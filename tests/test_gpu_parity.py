@@ -1,0 +1,325 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by
+element, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_16673_b200 import binding as speca
+from paper_2607_16673_b200 import synth
+from gpu_util import DevProblem, TOL, TOL_FP32, oracle_commit, oracle_verify, rel_err
+
+pytestmark = pytest.mark.gpu
+
+ROUTES = [speca.ROUTE_SERIAL]
+
+
+def cpu(t):
+    return t.detach().cpu().numpy()
+
+
+def check_verify(prob, route, chain=False, tol=TOL_FP32, want_u=False, max_nodes=None):
+    dp = DevProblem(prob, route=route, want_u=want_u, max_nodes=max_nodes)
+    S_before = dp.S.clone()
+    o = dp.verify_chain() if chain else dp.verify_tree()
+    assert dp.status_value() == 0
+    assert torch.equal(dp.S, S_before), "verify must leave the committed state bitwise unchanged"
+    ref = oracle_verify(prob)
+    e = rel_err(cpu(o), ref)
+    assert e <= tol and e <= TOL, f"{prob.name}: verify error {e:.3e}"
+    return dp, ref
+
+
+# ---------------------------------------------------------------------------
+# configuration 1: tiny chain, also against decode steps
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("route", ROUTES)
+def test_cfg1_chain_verify_commit_and_decode(route):
+    prob = synth.config(1)
+    dp, ref = check_verify(prob, route, chain=True)
+    o_chain = dp.o.clone()
+    dp.o.fill_(float("nan"))
+    dp.verify_tree()
+    assert rel_err(cpu(dp.o), ref) <= TOL_FP32                   # single-path tree == chain
+    # commit the first two tokens
+    dp.commit()
+    assert dp.status_value() == 0
+    S_ref = oracle_commit(prob, prob.path_idx, prob.path_len)
+    assert rel_err(cpu(dp.S), S_ref) <= TOL_FP32
+    # the same tokens by single-token decode steps
+    d1 = speca.Dims(prob.L, 1, prob.H, prob.d_k, prob.d_v)
+    S = torch.from_numpy(prob.S0).cuda()
+    So = prob.S0.astype(np.float64)
+    for t in range(prob.T):
+        o = torch.empty(prob.L, 1, prob.H, prob.d_v, device="cuda")
+        speca.decode_step(d1, S, dp.q[:, t:t + 1].contiguous(), dp.k[:, t:t + 1].contiguous(),
+                          dp.v[:, t:t + 1].contiguous(), dp.alpha[:, t:t + 1].contiguous(),
+                          dp.beta[:, t:t + 1].contiguous(), o)
+        So, oo = oracle.decode_step(So, prob.q[:, t:t + 1], prob.k[:, t:t + 1], prob.v[:, t:t + 1],
+                                    prob.alpha[:, t:t + 1], prob.beta[:, t:t + 1])
+        assert rel_err(cpu(o), oo) <= TOL_FP32
+        assert rel_err(cpu(S), So) <= TOL_FP32
+        assert rel_err(cpu(o[:, 0]), cpu(o_chain[:, t])) <= TOL_FP32
+        if t == 1:
+            assert rel_err(cpu(S), cpu(dp.S)) <= TOL_FP32         # commit of 2 == 2 decode steps
+
+
+# ---------------------------------------------------------------------------
+# configuration 2: 24 layers x 16 heads, chain of 8, accepted length 0..8
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("route", ROUTES)
+@pytest.mark.parametrize("accepted", [None, 0, 8])
+def test_cfg2_chain(route, accepted):
+    prob = synth.config(2)
+    if accepted is not None:
+        synth._set_paths(prob, [list(range(accepted))])
+    dp, _ = check_verify(prob, route, chain=True)
+    S_before = dp.S.clone()
+    dp.commit()
+    assert dp.status_value() == 0
+    if int(prob.path_len[0]) == 0:
+        assert torch.equal(dp.S, S_before)
+    S_ref = oracle_commit(prob, prob.path_idx, prob.path_len)
+    assert rel_err(cpu(dp.S), S_ref) <= TOL_FP32
+
+
+def test_cfg2_chain_equals_eight_decode_steps():
+    prob = synth.config(2)
+    dp = DevProblem(prob, route=speca.ROUTE_SERIAL)
+    o_chain = cpu(dp.verify_chain()).copy()
+    d1 = speca.Dims(prob.L, 1, prob.H, prob.d_k, prob.d_v)
+    S = dp.S.clone()
+    for t in range(8):
+        o = torch.empty(prob.L, 1, prob.H, prob.d_v, device="cuda")
+        speca.decode_step(d1, S, dp.q[:, t:t + 1].contiguous(), dp.k[:, t:t + 1].contiguous(),
+                          dp.v[:, t:t + 1].contiguous(), dp.alpha[:, t:t + 1].contiguous(),
+                          dp.beta[:, t:t + 1].contiguous(), o)
+        assert rel_err(cpu(o[:, 0]), o_chain[:, t]) <= TOL_FP32
+    synth._set_paths(prob, [list(range(8))])
+    dp2 = DevProblem(prob, route=speca.ROUTE_SERIAL)
+    dp2.commit()
+    assert rel_err(cpu(dp2.S), cpu(S)) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# configuration 3: 32-node tree, random root-to-leaf path committed
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("route", ROUTES)
+def test_cfg3_tree(route):
+    prob = synth.config(3)
+    dp, _ = check_verify(prob, route, want_u=True)
+    dp.commit()
+    assert dp.status_value() == 0
+    S_ref = oracle_commit(prob, prob.path_idx, prob.path_len)
+    assert rel_err(cpu(dp.S), S_ref) <= TOL_FP32
+    # u is the WY-style factor: S_t = gamma_t S0 + sum (gamma_t/gamma_i) u_i k_i^T rebuilds the committed state
+    l, h = 3, 5
+    path = prob.path_idx[0, :prob.path_len[0]]
+    S = prob.S0[l, 0, h].astype(np.float64)
+    u = cpu(dp.u)[l, :, h].astype(np.float64)
+    kf = synth.bf16_bits_to_f32(prob.k[l, :, h]).astype(np.float64)
+    for t in path:
+        S = prob.alpha[l, t, h].astype(np.float64) * S + np.outer(u[t], kf[t])
+    assert rel_err(S, S_ref[l, 0, h]) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# configuration 4 (reduced layers, full batch of ragged trees): verify -> accept -> commit
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("route", ROUTES)
+def test_cfg4_reduced_full_compare(route):
+    prob = synth.config(4, L=2)
+    dp, _ = check_verify(prob, route)
+    dp.accept()
+    pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                      prob.root_target_tok, prob.max_depth)
+    assert dp.status_value() == 0
+    assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+    assert np.array_equal(cpu(dp.next_tok), nt)
+    assert pl.max() >= 2
+    dp.commit()
+    assert dp.status_value() == 0
+    assert rel_err(cpu(dp.S), oracle_commit(prob, pi, pl)) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# shapes: every supported d_k, several d_v, tiles with ragged tails
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("d_k,d_v", [(64, 32), (64, 96), (128, 160), (256, 64), (256, 256), (128, 1024)])
+def test_shapes(d_k, d_v):
+    rng = np.random.default_rng(d_k + d_v)
+    parents = [synth.random_tree_parent(19, 6, 3, rng), synth.chain_parent(5), synth.random_tree_parent(33, 8, 4, rng)]
+    prob = synth.make_problem(d_k * 7 + d_v, 2, 3, d_k, d_v, parents, state_std=0.5, name=f"shape{d_k}x{d_v}")
+    prob.scale = 0.125
+    dp, _ = check_verify(prob, speca.ROUTE_SERIAL, want_u=True)
+    dp.accept()
+    pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                      prob.root_target_tok, prob.max_depth)
+    assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+    dp.commit()
+    assert rel_err(cpu(dp.S), oracle_commit(prob, pi, pl)) <= TOL_FP32
+    # decode step on the same shapes
+    L, B, H = prob.L, prob.B, prob.H
+    q, k, v, al, be = synth.draw_records(rng, L, B, H, d_k, d_v)
+    d1 = speca.Dims(L, B, H, d_k, d_v, scale=0.125)
+    from gpu_util import bf16_dev
+    S = torch.from_numpy(prob.S0).cuda()
+    o = torch.empty(L, B, H, d_v, device="cuda")
+    speca.decode_step(d1, S, bf16_dev(q), bf16_dev(k), bf16_dev(v), torch.from_numpy(al).cuda(),
+                      torch.from_numpy(be).cuda(), o)
+    Sr, orf = oracle.decode_step(prob.S0, q, k, v, al, be, scale=0.125)
+    assert rel_err(cpu(S), Sr) <= TOL_FP32 and rel_err(cpu(o), orf) <= TOL_FP32
+
+
+# ---------------------------------------------------------------------------
+# edge cases
+# ---------------------------------------------------------------------------
+def test_empty_sequences_single_nodes_and_forests():
+    rng = np.random.default_rng(77)
+    forest = np.array([-1, -1, 0, -1, 1, 1, 2, 3, 3, 6], np.int32)       # three roots
+    stars = np.array([-1] * 6, np.int32)                                   # "all-root" proposal
+    parents = [np.zeros(0, np.int32), synth.chain_parent(1), forest, np.zeros(0, np.int32), stars,
+               synth.random_tree_parent(64, 8, 4, rng)]
+    prob = synth.make_problem(78, 2, 2, 128, 64, parents, state_std=0.3)
+    dp, _ = check_verify(prob, speca.ROUTE_SERIAL)
+    dp.accept()
+    pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                      prob.root_target_tok, prob.max_depth)
+    assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+    assert np.array_equal(cpu(dp.next_tok), nt)
+    assert pl[0] == 0 and pl[3] == 0
+    S_before = dp.S.clone()
+    dp.commit()
+    assert dp.status_value() == 0
+    assert rel_err(cpu(dp.S), oracle_commit(prob, pi, pl)) <= TOL_FP32
+    for b in np.flatnonzero(pl == 0):
+        assert torch.equal(dp.S[:, int(b)], S_before[:, int(b)])
+
+
+def test_maximum_depth_and_node_budget():
+    rng = np.random.default_rng(5)
+    parents = [synth.chain_parent(16), synth.random_tree_parent(200, 16, 4, rng)]
+    prob = synth.make_problem(6, 1, 2, 64, 64, parents, max_depth=16, state_std=0.2)
+    synth._set_paths(prob, [list(range(16)), synth.root_path(parents[1], 199)])
+    dp, _ = check_verify(prob, speca.ROUTE_SERIAL)
+    dp.commit()
+    assert dp.status_value() == 0
+    assert rel_err(cpu(dp.S), oracle_commit(prob, prob.path_idx, prob.path_len)) <= TOL_FP32
+
+
+def test_device_side_faults_set_status_and_skip_the_sequence():
+    rng = np.random.default_rng(9)
+    parents = [synth.random_tree_parent(12, 5, 3, rng) for _ in range(4)]
+    prob = synth.make_problem(10, 1, 2, 64, 64, parents)
+    good = oracle_verify(prob)
+    s1, e1 = int(prob.node_offsets[1]), int(prob.node_offsets[2])
+    # (a) forward parent pointer in sequence 1
+    bad = synth.make_problem(10, 1, 2, 64, 64, parents)
+    bad.parent[s1 + 3] = 7
+    dp = DevProblem(bad, route=speca.ROUTE_SERIAL)
+    dp.verify_tree(with_depth=False)
+    assert dp.status_value() & speca.STATUS_BAD_PARENT
+    o = cpu(dp.o)
+    assert np.all(np.isnan(o[:, s1:e1]))                               # skipped: outputs untouched
+    keep = np.r_[0:s1, e1:prob.T]
+    assert rel_err(o[:, keep], good[:, keep]) <= TOL_FP32
+    dp.status.zero_()
+    dp.accept()
+    assert dp.status_value() & speca.STATUS_BAD_PARENT and int(dp.path_len[1]) == 0
+    # (b) node budget exceeded
+    dp = DevProblem(prob, route=speca.ROUTE_SERIAL, max_nodes=12)
+    dp.dims.max_nodes = 11
+    dp.verify_tree()
+    assert dp.status_value() & speca.STATUS_TOO_MANY
+    assert np.all(np.isnan(cpu(dp.o)))
+    # (c) deeper than max_depth
+    deep = synth.make_problem(11, 1, 1, 64, 64, [synth.chain_parent(6)], max_depth=4)
+    dp = DevProblem(deep, route=speca.ROUTE_SERIAL)
+    dp.verify_tree()
+    assert dp.status_value() & speca.STATUS_TOO_DEEP
+    # (d) inconsistent depth[] is reported
+    dp = DevProblem(prob, route=speca.ROUTE_SERIAL)
+    dp.depth[2] += 1
+    dp.verify_tree()
+    assert dp.status_value() & speca.STATUS_BAD_DEPTH
+    # (e) commit: path that is not a parent chain, and over-long path: state untouched
+    dp = DevProblem(prob, route=speca.ROUTE_SERIAL)
+    S0 = dp.S.clone()
+    leaf = synth.root_path(parents[2], 11)
+    idx = np.full((4, 8), -1, np.int32); ln = np.zeros(4, np.int32)
+    idx[2, :len(leaf)] = leaf[::-1]; ln[2] = len(leaf)                   # reversed: not a chain from a root
+    idx[0, :1] = [0]; ln[0] = 1
+    dp.path_idx.copy_(torch.from_numpy(idx)); dp.path_len.copy_(torch.from_numpy(ln))
+    dp.commit()
+    assert dp.status_value() & speca.STATUS_BAD_PATH
+    assert torch.equal(dp.S[:, 2], S0[:, 2]) and torch.equal(dp.S[:, 1], S0[:, 1])
+    assert not torch.equal(dp.S[:, 0], S0[:, 0])
+    dp.status.zero_()
+    ln[:] = 0; ln[3] = 9
+    dp.path_len.copy_(torch.from_numpy(ln))
+    S1 = dp.S.clone()
+    dp.commit()
+    assert dp.status_value() & speca.STATUS_TOO_DEEP and torch.equal(dp.S, S1)
+
+
+def test_outputs_stay_inside_their_buffers():
+    """Guard bands around o and S: nothing outside the tensors is written."""
+    prob = synth.config(3, L=2)
+    dp = DevProblem(prob, route=speca.ROUTE_SERIAL)
+    n = dp.o.numel()
+    big = torch.full((n + 512,), 7.5, device="cuda")
+    dp.o = big[256:256 + n].view_as(dp.o)
+    dp.verify_tree()
+    torch.cuda.synchronize()
+    assert torch.all(big[:256] == 7.5) and torch.all(big[-256:] == 7.5)
+    ns = dp.S.numel()
+    bigS = torch.full((ns + 512,), 7.5, device="cuda")
+    bigS[256:256 + ns] = dp.S.flatten()
+    dp.S = bigS[256:256 + ns].view_as(dp.S)
+    dp.commit()
+    torch.cuda.synchronize()
+    assert torch.all(bigS[:256] == 7.5) and torch.all(bigS[-256:] == 7.5)
+    assert dp.status_value() == 0
+
+
+def test_accept_matches_oracle_on_many_random_batches():
+    rng = np.random.default_rng(123)
+    for trial in range(6):
+        parents = synth.ragged_tree_batch(rng, 40, 1, 64, 8)
+        prob = synth.make_problem(200 + trial, 1, 1, 64, 32, parents, p_match=0.85)
+        dp = DevProblem(prob)
+        dp.accept()
+        pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                          prob.root_target_tok, prob.max_depth)
+        assert dp.status_value() == 0
+        assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+        assert np.array_equal(cpu(dp.next_tok), nt)
+
+
+def test_multi_round_loop_carries_state():
+    """verify -> accept -> commit for several rounds with fresh drafts, the oracle carrying its own fp64 state."""
+    rng = np.random.default_rng(31)
+    L, B, H, dk, dv = 2, 6, 2, 128, 256
+    S_ref = None
+    S_dev = None
+    for rnd in range(4):
+        parents = synth.mixed_chain_tree_batch(rng, B, 8, 40, 8)
+        prob = synth.make_problem(300 + rnd, L, H, dk, dv, parents, p_match=0.9)
+        if S_ref is None:
+            S_ref = prob.S0.astype(np.float64)
+        dp = DevProblem(prob, route=speca.ROUTE_SERIAL)
+        if S_dev is not None:
+            dp.S.copy_(S_dev)
+        o = dp.verify_tree()
+        o_ref = oracle.verify_tree(S_ref, prob.q, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets,
+                                   prob.parent)
+        assert rel_err(cpu(o), o_ref) <= TOL_FP32 * (rnd + 1)
+        dp.accept()
+        pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                          prob.root_target_tok, prob.max_depth)
+        assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+        dp.commit()
+        S_ref = oracle.commit(S_ref, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets, pi, pl)
+        assert rel_err(cpu(dp.S), S_ref) <= TOL_FP32 * (rnd + 1)
+        assert dp.status_value() == 0
+        S_dev = dp.S.clone()
