@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative verify -> accept -> commit path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4] [--impl reference]
+
+One "step" is one round of the whole hot path over one batch of synthetic draft input:
+plan + verify (all layers, heads, nodes) -> greedy accept -> commit, with the committed
+state carried from step to step.  The default workload is the largest single-GPU
+configuration: 128 sequences, 24 layers, 16 heads, d_k = 128, d_v = 256, half of the
+sequences with 8-token chains and half with 64-node trees.
+
+The metric is verified draft token-layers per second (tokens verified in one step times
+the layer count, divided by the step time).  Rank 0 prints ONE JSON line.  For N > 1 the
+sequences are partitioned over the ranks (every rank owns whole sequences; there is no
+exchange step anywhere on the path), launched one process per GPU by torchrun.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified draft token-layers/s (verify+accept+commit)"
+UNIT = "token-layers/s"
+
+WORKLOADS = {
+    # name: (L, B, H, d_k, d_v, description)
+    "cfg5": (24, 128, 16, 128, 256, "128 seq x 24 layers x 16 heads, d_k=128 d_v=256; 64 seq with 8-token chains + "
+                                    "64 seq with 64-node trees (depth<=8)"),
+    "cfg4": (24, 32, 16, 128, 256, "32 seq x 24 layers x 16 heads, d_k=128 d_v=256; ragged trees of 8..64 nodes (depth<=8)"),
+}
+POOL = 3            # independent draft inputs rotated over the steps ("fresh draft factors each round")
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
+    ap.add_argument("--route", type=int, default=0, help="0 auto, 1 serial, 2 factorized")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling only)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling only)")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------
+# workload description (host side: topology and token ids; no method arithmetic)
+# ---------------------------------------------------------------------------
+def host_round_inputs(name: str, B: int, seed: int):
+    """Topology and token ids of one round, on the host."""
+    from paper_2607_16673_b200 import synth
+    rng = np.random.default_rng(seed)
+    if name == "cfg5":
+        parents = synth.mixed_chain_tree_batch(rng, B, 8, 64, 8)
+    else:
+        parents = synth.ragged_tree_batch(rng, B, 8, 64, 8)
+    sizes = [len(p) for p in parents]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    parent = np.concatenate(parents).astype(np.int32)
+    depth = np.concatenate([synth.depth_of(p) for p in parents]).astype(np.int32)
+    draft, target, root_target = synth.draw_tokens(rng, offs, parent, 0.75)
+    return dict(parents=parents, node_offsets=offs, parent=parent, depth=depth, draft_tok=draft,
+                target_tok=target, root_target_tok=root_target, T=int(offs[-1]))
+
+
+def algorithmic_bytes(L, B, H, dk, dv, T, path_len):
+    """Bytes the method itself must move in one step (HBM roofline numerator)."""
+    units = L * B * H
+    Sb = 4 * dk * dv
+    rec_in = 4 * dk + 2 * dv + 8             # q, k bf16 + v bf16 + alpha, beta fp32 per node per (layer, head)
+    verify = units * Sb + T * L * H * rec_in + T * L * H * 4 * dv
+    n_commit_seq = int(np.count_nonzero(path_len))
+    commit = 2 * n_commit_seq * L * H * Sb + int(path_len.sum()) * L * H * (2 * dk + 2 * dv + 8)
+    return verify, commit
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------
+def run_speca(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_16673_b200 import binding as speca
+    from paper_2607_16673_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    L, B, H, dk, dv, desc = WORKLOADS[args.workload]
+    L = args.layers or L
+    B = args.batch or B
+    dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, args.route)
+    stream = torch.cuda.current_stream()
+
+    # --- inputs resident in HBM -------------------------------------------------
+    S = synth.device_state(1000 + rank, L, B, H, dk, dv, 0.02, dev)
+    pool = []
+    for j in range(POOL):
+        hi = host_round_inputs(args.workload, B, 5000 + 97 * rank + j)
+        q, k, v, al, be = synth.device_records(7000 + 97 * rank + j, L, hi["T"], H, dk, dv, dev)
+        t = lambda a: torch.from_numpy(a).to(dev)
+        pool.append(dict(hi, q=q, k=k, v=v, alpha=al, beta=be, d_offs=t(hi["node_offsets"]),
+                         d_parent=t(hi["parent"]), d_depth=t(hi["depth"]), d_draft=t(hi["draft_tok"]),
+                         d_target=t(hi["target_tok"]), d_root=t(hi["root_target_tok"])))
+    Tmax = max(p["T"] for p in pool)
+    o_buf = torch.empty(L * Tmax * H * dv, dtype=torch.float32, device=dev)
+    ws = speca.alloc_workspace(dims, Tmax, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    path_idx = torch.zeros(B, 8, dtype=torch.int32, device=dev)
+    path_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    next_tok = torch.zeros(B, dtype=torch.int32, device=dev)
+
+    def o_view(T):
+        return o_buf[: L * T * H * dv].view(L, T, H, dv)
+
+    def step(p, ev=None):
+        T = p["T"]
+        if ev: ev[0].record(stream)
+        speca.verify_tree(dims, S, p["q"], p["k"], p["v"], p["alpha"], p["beta"], p["d_offs"], T, p["d_parent"],
+                          p["d_depth"], o_view(T), None, ws, status)
+        if ev: ev[1].record(stream)
+        speca.greedy_accept(B, 8, p["d_offs"], p["d_parent"], p["d_draft"], p["d_target"], p["d_root"],
+                            path_idx, path_len, next_tok, status)
+        if ev: ev[2].record(stream)
+        speca.commit(dims, S, p["k"], p["v"], p["alpha"], p["beta"], p["d_offs"], T, p["d_parent"], path_idx,
+                     path_len, status)
+        if ev: ev[3].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # accepted lengths per pool entry (integer-only, independent of the state): for the byte counts
+    for p in pool:
+        speca.greedy_accept(B, 8, p["d_offs"], p["d_parent"], p["d_draft"], p["d_target"], p["d_root"],
+                            path_idx, path_len, next_tok, status)
+        torch.cuda.synchronize()
+        p["path_len"] = path_len.cpu().numpy().copy()
+
+    for w in range(args.warmup):
+        step(pool[w % POOL])
+    barrier()
+
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_start.record(stream)
+    for i in range(K):
+        step(pool[(args.warmup + i) % POOL], evs[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = t_start.elapsed_time(t_end)
+    assert int(status.item()) == 0, f"device status word {int(status.item())}"
+
+    tokens = sum(pool[(args.warmup + i) % POOL]["T"] for i in range(K))
+    vb = cb = 0
+    for i in range(K):
+        p = pool[(args.warmup + i) % POOL]
+        a, c = algorithmic_bytes(L, B, H, dk, dv, p["T"], p["path_len"])
+        vb += a; cb += c
+    t_verify = sum(e[0].elapsed_time(e[1]) for e in evs) / K       # plan + verify kernels
+    t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / K
+    t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / K
+
+    if world > 1:
+        tt = torch.tensor([total_ms, t_verify, t_commit], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, t_verify, t_commit = (float(x) for x in tt.tolist())
+        cnt = torch.tensor([tokens, vb, cb], device=dev, dtype=torch.float64)
+        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
+        tokens_all = float(cnt[0]); vb_all = float(cnt[1]); cb_all = float(cnt[2])
+    else:
+        tokens_all, vb_all, cb_all = float(tokens), float(vb), float(cb)
+
+    # --- decode-step baseline at the same batch (context) --------------------------
+    q1, k1, v1, a1, b1 = synth.device_records(99, L, B, H, dk, dv, dev)
+    o1 = torch.empty(L, B, H, dv, device=dev)
+    d1 = speca.Dims(L, B, H, dk, dv)
+    S_dec = S.clone() if S.numel() * 4 < 20e9 else S
+    for _ in range(2):
+        speca.decode_step(d1, S_dec, q1, k1, v1, a1, b1, o1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    n_dec = 5
+    for _ in range(n_dec):
+        speca.decode_step(d1, S_dec, q1, k1, v1, a1, b1, o1)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    dec_ms = e0.elapsed_time(e1) / n_dec
+    dec_bytes = L * B * H * (2 * 4 * dk * dv + 4 * dk + 2 * dv + 8 + 4 * dv)
+    del S_dec
+
+    # --- end to end with host buffers (C ABI fed from pinned host memory) ---------
+    e2e = None
+    if not args.no_e2e and rank == 0:
+        e2e = run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream)
+    if world > 1:
+        dist.barrier()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peak_gbs()
+    ms_per_step = total_ms / K
+    value = tokens_all * L / (total_ms * 1e-3)
+    dom = "verify" if t_verify >= t_commit else "commit"
+    dom_ms = max(t_verify, t_commit)
+    dom_bytes = (vb if dom == "verify" else cb) / K
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {desc}", "n_layers": L, "batch_per_gpu": B, "heads": H,
+                   "d_k": dk, "d_v": dv, "nodes_per_step_per_gpu": [p["T"] for p in pool],
+                   "mean_accepted_len": float(np.mean([p["path_len"].mean() for p in pool])),
+                   "input_pool": POOL, "l2": "inputs larger than L2 (state 6.4 GB, records 1.8 GB per round at full size)",
+                   "route": args.route, "parallelism": f"dp{world} (sequences partitioned, no collective)"},
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get(dom),
+                     "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms},
+        "kernels": {"verify_ms": t_verify, "accept_ms": t_accept, "commit_ms": t_commit,
+                    "verify_gbs": vb / K / (t_verify * 1e-3) / 1e9, "commit_gbs": cb / K / (t_commit * 1e-3) / 1e9,
+                    "step_gbs": (vb + cb) / K / (ms_per_step * 1e-3) / 1e9,
+                    "step_frac_of_peak": (vb + cb) / K / (ms_per_step * 1e-3) / 1e9 / peak,
+                    "step_frac_of_8TBs": (vb + cb) / K / (ms_per_step * 1e-3) / 1e9 / 8000.0},
+        "decode_step": {"ms": dec_ms, "gbs": dec_bytes / (dec_ms * 1e-3) / 1e9,
+                        "token_layers_per_s": B * L / (dec_ms * 1e-3),
+                        "note": "one autoregressive token per sequence at the same batch"},
+        "gpu_launches": 4 * K,
+        "clocks": clocks,
+        "e2e": e2e,
+    }
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(args.workload, L, H, dk, dv)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant
+# kernels from the ncu captures summarised under profiles/; None until captured.
+NCU_TRAFFIC = {"verify": None, "commit": None}
+
+
+def run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream):
+    """Same step, but every step's draft inputs start in pinned HOST memory and its results
+    (outputs o, accepted paths, next tokens) are read back to the host inside the timed region.
+    The committed state is the durable device-resident object and stays in HBM."""
+    import torch
+    L, B, H, dk, dv = dims.n_layers, dims.batch, dims.heads, dims.d_k, dims.d_v
+    p0 = pool[0]
+    T = p0["T"]
+    names = ["q", "k", "v", "alpha", "beta", "d_offs", "d_parent", "d_depth", "d_draft", "d_target", "d_root"]
+    host = {n: torch.empty(p0[n].shape, dtype=p0[n].dtype, pin_memory=True).copy_(p0[n]) for n in names}
+    devb = {n: torch.empty_like(p0[n]) for n in names}
+    o = o_buf[: L * T * H * dv].view(L, T, H, dv)
+    o_host = torch.empty(o.shape, dtype=o.dtype, pin_memory=True)
+    pi_host = torch.empty(path_idx.shape, dtype=torch.int32, pin_memory=True)
+    pl_host = torch.empty(path_len.shape, dtype=torch.int32, pin_memory=True)
+    nt_host = torch.empty(next_tok.shape, dtype=torch.int32, pin_memory=True)
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = sum(x.numel() * x.element_size() for x in (o_host, pi_host, pl_host, nt_host))
+
+    def one():
+        for n in names:
+            devb[n].copy_(host[n], non_blocking=True)
+        speca.verify_tree(dims, S, devb["q"], devb["k"], devb["v"], devb["alpha"], devb["beta"], devb["d_offs"], T,
+                          devb["d_parent"], devb["d_depth"], o, None, ws, status)
+        speca.greedy_accept(B, 8, devb["d_offs"], devb["d_parent"], devb["d_draft"], devb["d_target"], devb["d_root"],
+                            path_idx, path_len, next_tok, status)
+        speca.commit(dims, S, devb["k"], devb["v"], devb["alpha"], devb["beta"], devb["d_offs"], T, devb["d_parent"],
+                     path_idx, path_len, status)
+        o_host.copy_(o, non_blocking=True)
+        pi_host.copy_(path_idx, non_blocking=True)
+        pl_host.copy_(path_len, non_blocking=True)
+        nt_host.copy_(next_tok, non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = max(1, args.e2e_steps)
+    e0.record(stream)
+    for _ in range(n):
+        one()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    return {"value": T * L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": n,
+            "note": "draft inputs from pinned host memory, outputs and accepted paths read back; state stays in HBM"}
+
+
+# ---------------------------------------------------------------------------
+# the oracle on the host cores (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------
+def oracle_sample_problem(workload: str, H: int, dk: int, dv: int, n_units: int, seed: int = 4242):
+    """A bounded sample of the workload: n_units (layer, sequence, head) units, half chains and half
+    trees for cfg5 (ragged trees for cfg4), repacked as independent single-head sequences."""
+    from paper_2607_16673_b200 import synth
+    rng = np.random.default_rng(seed)
+    if workload == "cfg5":
+        parents = synth.mixed_chain_tree_batch(rng, n_units, 8, 64, 8)
+    else:
+        parents = synth.ragged_tree_batch(rng, n_units, 8, 64, 8)
+    return synth.make_problem(seed, 1, 1, dk, dv, parents)
+
+
+def time_oracle_once(prob):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.verify_tree(prob.S0, prob.q, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets, prob.parent)
+    pi, pl, nt = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                      prob.root_target_tok, prob.max_depth)
+    oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets, pi, pl)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(workload: str, L: int, H: int, dk: int, dv: int, n_units: int = 1536):
+    import oracle
+    prob = oracle_sample_problem(workload, H, dk, dv, n_units)
+    time_oracle_once(oracle_sample_problem(workload, H, dk, dv, 8))      # build + page in
+    dt = time_oracle_once(prob)
+    # one unit is 1/H of a token-layer
+    value = prob.T / H / dt
+    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n_units} (layer, sequence, head) units of {workload} ({prob.T} node-units), "
+                      f"verify+accept+commit in {dt:.2f} s, scaled by 1/heads to token-layers"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    L, B, H, dk, dv, desc = WORKLOADS[args.workload]
+    n_units = 192
+    prob = oracle_sample_problem(args.workload, H, dk, dv, n_units)
+    for _ in range(max(1, min(args.warmup, 3))):
+        time_oracle_once(oracle_sample_problem(args.workload, H, dk, dv, 8))
+    K = args.steps
+    t = 0.0
+    for _ in range(K):
+        t += time_oracle_once(prob)
+    value = K * prob.T / H / t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+        "warmup": args.warmup, "ms_per_step": t / K * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {desc}", "sample_units_per_step": n_units},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"each step: {n_units} (layer, sequence, head) units of {args.workload} "
+                                   f"({prob.T} node-units), scaled by 1/heads to token-layers"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_speca(args)
+
+
+if __name__ == "__main__":
+    main()

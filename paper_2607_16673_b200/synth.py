@@ -299,3 +299,36 @@ def gather_units(prob: Problem, units: Sequence[tuple]) -> Problem:
         sub.path_idx = np.stack([prob.path_idx[b] for (_, b, _) in units]).astype(np.int32)
         sub.path_len = np.asarray([prob.path_len[b] for (_, b, _) in units], dtype=np.int32)
     return sub
+
+
+# ----------------------------------------------------------------------------
+# on-device drawing for the multi-GB configurations (same distributions, torch RNG)
+# ----------------------------------------------------------------------------
+def device_state(seed: int, L: int, B: int, H: int, d_k: int, d_v: int, std: float = 0.02, device="cuda"):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    S = torch.empty((L, B, H, d_v, d_k), dtype=torch.float32, device=device)
+    for l in range(L):                       # layer by layer: no multi-GB temporaries
+        S[l].normal_(0.0, std, generator=g)
+    return S
+
+
+def device_records(seed: int, L: int, T: int, H: int, d_k: int, d_v: int, device="cuda"):
+    """q, k, v (bf16), alpha, beta (fp32) with the distributions of ``draw_records``."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    q = torch.empty((L, T, H, d_k), dtype=torch.bfloat16, device=device)
+    k = torch.empty((L, T, H, d_k), dtype=torch.bfloat16, device=device)
+    v = torch.empty((L, T, H, d_v), dtype=torch.bfloat16, device=device)
+    for l in range(L):
+        q[l] = torch.randn((T, H, d_k), generator=g, device=device)
+        kk = torch.randn((T, H, d_k), generator=g, device=device)
+        k[l] = kk / kk.norm(dim=-1, keepdim=True)
+        v[l] = torch.randn((T, H, d_v), generator=g, device=device)
+    xb = torch.randn((L, T, H), generator=g, device=device, dtype=torch.float64)
+    xa = torch.randn((L, T, H), generator=g, device=device, dtype=torch.float64)
+    beta = torch.sigmoid(xb).float()
+    alpha = torch.sigmoid(-xa).float()
+    return q, k, v, alpha, beta

@@ -226,12 +226,18 @@ def test_device_side_faults_set_status_and_skip_the_sequence():
     dp.status.zero_()
     dp.accept()
     assert dp.status_value() & speca.STATUS_BAD_PARENT and int(dp.path_len[1]) == 0
-    # (b) node budget exceeded
-    dp = DevProblem(prob, route=speca.ROUTE_SERIAL, max_nodes=12)
-    dp.dims.max_nodes = 11
+    # (b) node budget exceeded by one sequence only: that sequence is skipped, the rest is computed
+    big = synth.make_problem(12, 1, 2, 64, 64, [parents[0], synth.random_tree_parent(20, 5, 3, rng), parents[2]])
+    dp = DevProblem(big, route=speca.ROUTE_SERIAL, max_nodes=16)
     dp.verify_tree()
     assert dp.status_value() & speca.STATUS_TOO_MANY
-    assert np.all(np.isnan(cpu(dp.o)))
+    o, ref = cpu(dp.o), oracle_verify(big)
+    assert np.all(np.isnan(o[:, 12:32]))
+    keep = np.r_[0:12, 32:44]
+    assert rel_err(o[:, keep], ref[:, keep]) <= TOL_FP32
+    dp.o.fill_(float("nan")); dp.status.zero_()
+    dp.verify_chain()                                   # the chain entry point applies the same budget
+    assert dp.status_value() & speca.STATUS_TOO_MANY and np.all(np.isnan(cpu(dp.o)[:, 12:32]))
     # (c) deeper than max_depth
     deep = synth.make_problem(11, 1, 1, 64, 64, [synth.chain_parent(6)], max_depth=4)
     dp = DevProblem(deep, route=speca.ROUTE_SERIAL)
