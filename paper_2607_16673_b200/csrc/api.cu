@@ -63,10 +63,15 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
     p.status = status_word;
     p.ws = carve_workspace(workspace, dims->batch, total_nodes);
     p.n_slots = tree_slots_needed(dims->max_nodes);
-    if (!chain) {
+    const bool can_factorize = factorized_supported(dims);
+    if (dims->route == SPECA_ROUTE_FACTORIZED && !can_factorize) return SPECA_ERR_UNSUPPORTED;
+    const bool factorize = can_factorize && dims->route != SPECA_ROUTE_SERIAL;
+    if (!chain || factorize) {
+        // with parent == NULL (chain entry point) the plan kernel assumes parent[i] = i - 1
         rc = cuda_rc(launch_plan(p, st));
         if (rc != SPECA_OK) return rc;
     }
+    if (factorize) return cuda_rc(launch_verify_factorized(p, st));
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 

@@ -16,7 +16,7 @@ namespace {
 
 constexpr int kPlanThreads = 128;
 
-// One CTA per sequence.  Dynamic smem: 5 int32 arrays of max_nodes (+1).
+// One CTA per sequence.  Dynamic smem: 6 int32 arrays of max_nodes (+1).
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict__ parent,
             const int32_t *__restrict__ depth_in, int32_t B, int32_t T, int32_t max_depth,
@@ -44,13 +44,14 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
     int32_t *bef = size + max_nodes;         // [n]   total size of siblings visited before this node
     int32_t *nlc = bef + max_nodes;          // [n+1] children with children, index shifted by one (slot 0 = committed state)
     int32_t *ldf = nlc + max_nodes + 1;      // [n]   1 if an earlier sibling has children (register state lost)
+    int32_t *posn = ldf + max_nodes;         // [n]   position of node i in the processing order
 
     if (tid == 0) s_flag = 0;
     for (int i = tid; i < n; i += kPlanThreads) { size[i] = 0; nlc[i + 1] = 0; }
     if (tid == 0) nlc[0] = 0;
     __syncthreads();
     for (int i = tid; i < n; i += kPlanThreads) {
-        int p = parent[base + i];
+        int p = parent != nullptr ? parent[base + i] : i - 1;      // no parent array: chain
         par[i] = p;
         if (p < -1 || p >= i) atomicOr(&s_flag, SPECA_STATUS_BAD_PARENT);
     }
@@ -107,6 +108,29 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
         }
         if (leaf) entry |= kPlanLeafBit;
         ws.plan[base + pos] = entry;
+        posn[i] = pos;
+    }
+    __syncthreads();
+    // Per position: depth, node index and the positions of the node's ancestors by depth
+    // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 8, which is
+    // all the factorised route accepts).
+    for (int i = tid; i < n; i += kPlanThreads) {
+        int d = 0;
+        for (int a = i; a >= 0; a = par[a]) ++d;
+        uint32_t lo = 0, hi = 0;
+        int j = d - 1;
+        for (int a = par[i]; a >= 0; a = par[a]) {
+            --j;
+            const uint32_t byte = uint32_t(posn[a]) & 0xffu;
+            if (j < 4) lo |= byte << (8 * j);
+            else if (j < 8) hi |= byte << (8 * (j - 4));
+        }
+        int4 rec;
+        rec.x = d | (i << 8);
+        rec.y = int(lo);
+        rec.z = int(hi);
+        rec.w = 0;
+        reinterpret_cast<int4 *>(ws.anc)[base + posn[i]] = rec;
     }
     __syncthreads();
     if (tid == 0) {
@@ -172,7 +196,7 @@ accept_kernel(int32_t B, int32_t max_depth, const int32_t *__restrict__ node_off
 
 int launch_plan(const Params &p, cudaStream_t st)
 {
-    const size_t smem = size_t(5 * p.max_nodes + 1) * sizeof(int32_t);
+    const size_t smem = size_t(6 * p.max_nodes + 1) * sizeof(int32_t);
     plan_kernel<<<p.B, kPlanThreads, smem, st>>>(p.node_offsets, p.parent, p.depth_in, p.B, p.T,
                                                   p.max_depth, p.max_nodes, p.n_slots, p.ws, p.status);
     return int(cudaGetLastError());

@@ -15,7 +15,7 @@ namespace speca {
 //   [0, 256)                     control words (work-queue counters)
 //   [256, 256 + 4*Bpad)          seq_n[b]: node count of sequence b, or -1 if the
 //                                sequence failed validation and must be skipped
-//   then 4 int32 arrays of Tpad: plan[], depth[], anc_lo[], anc_hi[] ...
+//   then int32 arrays of Tpad words: plan[T], depth[T], anc[T][4]
 // Every region starts on a 256-byte boundary.
 // ---------------------------------------------------------------------------
 constexpr size_t kCtrlBytes = 256;
@@ -28,7 +28,7 @@ struct Workspace {
     int32_t *seq_n;     // [B]
     int32_t *plan;      // [T]   packed schedule entries, in processing order per sequence
     int32_t *depth;     // [T]   depth computed from parent[]
-    int32_t *anc;       // [T][kMaxDepthWords] reserved for the factorised route
+    int32_t *anc;       // [T][4] per processing position: depth | node << 8, ancestor positions (8 bytes), spare
 };
 
 inline size_t workspace_bytes(int32_t batch, int32_t total_nodes)
@@ -83,6 +83,8 @@ int launch_plan(const Params &p, cudaStream_t st);
 int launch_decode(const Params &p, int d_k, cudaStream_t st);
 int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
 int launch_commit(const Params &p, int d_k, cudaStream_t st);
+bool factorized_supported(const speca_dims *d);
+int launch_verify_factorized(const Params &p, cudaStream_t st);
 int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
                   const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
                   int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,
