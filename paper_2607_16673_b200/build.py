@@ -40,6 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"] + ARCH
     if verbose:
         flags += ["-Xptxas", "-v"]
+    flags += os.environ.get("SPECA_NVCC_FLAGS", "").split()
     objs = []
     procs = []
     for src in SOURCES:

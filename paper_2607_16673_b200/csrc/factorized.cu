@@ -19,12 +19,17 @@
 //   * [K;Q] of the sequence's nodes, converted bf16 -> fp32 (exact in TF32) and laid out in
 //     depth-first order, is the B operand; one MMA chain per tile gives D[v, node] =
 //     (R | G)^T in TMEM with value rows on TMEM lanes, so the substitution is thread-local;
-//   * the same [K;Q] block times K^T gives every q.k and k.k the coefficients need;
-//   * epilogue threads own one value row each, keep the u of the current depth-first path
-//     in registers (a stack indexed by depth) and stream o out coalesced.
+//   * the same [K;Q] block times K^T gives every q.k and k.k the coefficients need; that
+//     Gram block borrows the unit's own accumulator columns before the state MMAs start;
+//   * an epilogue thread owns one value row of EACH tile of the unit (same TMEM lane), so the
+//     per-node coefficients are fetched from shared memory once per two rows; it keeps the u
+//     of the current depth-first path in registers (a stack indexed by depth) and streams o
+//     out coalesced.
 // Roles: warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-5 operand/coefficient
-// preparation, warps 6-13 two epilogue groups.  Every wait is bounded; on expiry the CTA
-// raises SPECA_STATUS_TIMEOUT, drains and exits.
+// preparation, warps 6-9 and 10-13 two epilogue groups that alternate units.  Shared-memory
+// bandwidth (operand reads by the tensor core, coefficient broadcasts) is the scarce on-chip
+// resource, which is what the two-rows-per-thread epilogue is for.  Every wait is bounded; on
+// expiry the CTA raises SPECA_STATUS_TIMEOUT, drains and exits.
 #include <cuda.h>
 
 #include "speca_common.cuh"
@@ -43,23 +48,23 @@ constexpr int kMaxNodes = 64;                  // nodes per sequence handled by 
 constexpr int kMaxDepth = 8;
 constexpr int kBopRows = 2 * kMaxNodes;        // [K;Q] rows
 constexpr int kBopChunkBytes = kBopRows * 128; // 16 KiB per K-chunk region
-constexpr int kCoefStride = 20;                // floats per position: cU[8] cO[8] cV cR cG meta
-constexpr int kAccCols = 2 * kMaxNodes;        // 128 TMEM columns per accumulator
-constexpr int kNumAcc = 3;
-constexpr int kGramCol = kNumAcc * kAccCols;   // 384
-constexpr int kTmemCols = 512;
+constexpr int kCoefStride = 20;                // floats per position: cU[7] cV cO[8] cR cG depth-1 out-offset
+constexpr int kAccCols = 2 * kMaxNodes;        // 128 TMEM columns per tile accumulator (R | G)
+constexpr int kPairCols = 2 * kAccCols;        // a unit's two tiles
+constexpr int kTmemCols = 512;                 // two units in flight
 constexpr int kThreads = 14 * 32;
 constexpr int kPrepThreads = 128;
+constexpr int kEpiChunk = 4;                   // nodes per TMEM read in the epilogue
 constexpr int kGramHalf = 32;                  // Gram columns parked per extraction pass
-constexpr int kVBufBytes = kMaxNodes * kTileRows * 2;   // bf16 value tile of one sequence: 16 KiB
+constexpr int kStageChunkBytes = kBopRows * 128; // 64 bf16 columns of all [K;Q] rows: 16 KiB
 
 // shared memory carve-up (bytes, from a 1024-byte aligned base)
 constexpr int kOffRing = 0;
-constexpr int kOffBop = kOffRing + kStages * kStageBytes;                 // 98304
-constexpr int kOffGram = kOffBop + kChunks * kBopChunkBytes;              // +65536
-constexpr int kOffVBuf = kOffGram + kGramHalf * kTileRows * 4;            // +16384
-constexpr int kOffCoef = kOffVBuf + 2 * kVBufBytes;                       // +32768
-constexpr int kOffAlpha = kOffCoef + 2 * kMaxNodes * kCoefStride * 4;     // +10240
+constexpr int kOffBop = kOffRing + kStages * kStageBytes;
+constexpr int kOffStage = kOffBop + kChunks * kBopChunkBytes;              // raw bf16 [K;Q] rows of the next unit
+constexpr int kOffGram = kOffStage + 2 * kStageChunkBytes;
+constexpr int kOffCoef = kOffGram + kGramHalf * kTileRows * 4;
+constexpr int kOffAlpha = kOffCoef + 2 * kMaxNodes * kCoefStride * 4;
 constexpr int kOffBars = kOffAlpha + 2 * kMaxNodes * 4;                   // alpha, beta by position
 constexpr int kOffMisc = kOffBars + 8 * 32;
 constexpr int kSmemBytes = kOffMisc + 64 + 1024;                          // + alignment slack
@@ -70,14 +75,14 @@ enum Bar {
     kBarEmpty = kBarFull + kStages,      // [kStages] MMA -> TMA
     kBarBReady = kBarEmpty + kStages,    // prep -> MMA (and prep-internal): [K;Q] operand, alpha, beta written
     kBarBFree,                           // MMA -> prep: operand no longer read
+    kBarStageReady,                      // prep -> MMA: raw bf16 rows of a unit staged (Gram operand)
     kBarGramFull,                        // MMA -> prep: Gram block in TMEM
-    kBarCoefReady,                       // [2] prep -> epilogue
-    kBarCoefFree = kBarCoefReady + 2,    // [2] epilogue -> prep
-    kBarAccFull = kBarCoefFree + 2,      // [kNumAcc] MMA -> epilogue
-    kBarAccFree = kBarAccFull + kNumAcc, // [kNumAcc] epilogue -> MMA
-    kBarVReady = kBarAccFree + kNumAcc,  // [2] per epilogue group: staged value tile has landed
-    kBarVFree = kBarVReady + 2,          // [2] per epilogue group: staged value tile no longer read
-    kBarDrain = kBarVFree + 2,           // MMA warp: everything issued has completed
+    kBarGramDone,                        // prep -> MMA: Gram block read, its columns may be overwritten
+    kBarCoefReady,                       // [2] prep -> epilogue group
+    kBarCoefFree = kBarCoefReady + 2,    // [2] epilogue group -> prep
+    kBarAccFull = kBarCoefFree + 2,      // [2] MMA -> epilogue group: the unit's accumulators are complete
+    kBarPairFree = kBarAccFull + 2,      // [2] epilogue group -> MMA: accumulator columns released
+    kBarDrain = kBarPairFree + 2,        // MMA warp: everything issued has completed
     kBarCount
 };
 static_assert(kBarCount <= 32, "barrier region too small");
@@ -97,15 +102,11 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// the mbarrier receives one arrival once all earlier cp.async of this thread have landed
-__device__ __forceinline__ void cp_async_arrive(uint32_t bar)
-{
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -128,7 +129,7 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 // Bounded, warp-uniform wait.  Returns false if the CTA is aborting (this wait or another
 // one gave up); the caller must then leave its loop.  All 32 lanes must call it together.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;       // 2 s
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
     uint64_t t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -146,12 +147,53 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Optional self-profiling build (-DSPECA_PROF): cycles spent in each kind of wait per role.
+#ifdef SPECA_PROF
+#define PROF_DECL long long prof_w[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long prof_t0 = clock64(); long long prof_mark = prof_t0;
+#define PROF_MARK() prof_mark = clock64();
+#define PROF_SEG(slot) { const long long t_ = clock64(); prof_w[slot] += t_ - prof_mark; prof_mark = t_; }
+#define WAIT(slot, b, ph) prof_wait(prof_w[slot], b, ph, abort_flag)
+#define PROF_STORE()                                                                              \
+    if (blockIdx.x == 0 && lane == 0) {                                                           \
+        long long *dst = reinterpret_cast<long long *>(p.ws.ctrl) + 8 + warp * 9;                \
+        for (int i_ = 0; i_ < 8; ++i_) dst[i_] = prof_w[i_];                                      \
+        dst[8] = clock64() - prof_t0;                                                             \
+    }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag);
+__device__ __forceinline__ bool prof_wait(long long &acc, uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    const long long t = clock64();
+    const bool r = mbar_wait(bar, parity, abort_flag);
+    acc += clock64() - t;
+    return r;
+}
+#else
+#define PROF_DECL
+#define PROF_MARK()
+#define PROF_SEG(slot)
+#define WAIT(slot, b, ph) wait_fast(b, ph, abort_flag)
+#define PROF_STORE()
+#endif
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
 {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+// bring a box of a tensor into L2 ahead of the loads that will use it (no destination, no barrier)
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
+                 : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async()
 {
@@ -194,6 +236,16 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&r)[8])
 #pragma unroll
     for (int i = 0; i < 8; ++i) r[i] = __uint_as_float(x[i]);
 }
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, float (&r)[4])
+{
+    uint32_t x[4];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r[i] = __uint_as_float(x[i]);
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // K-major operand descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -213,48 +265,123 @@ __device__ __forceinline__ uint32_t make_idesc(int n)
     return (1u << 4) | (2u << 7) | (2u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(kTileRows >> 4) << 24);
 }
 
+// Tensor maps of the bf16 key / query records, view [L*T][H][d_k], one per box height
+// (16, 32, 48, 64 nodes): a unit's rows are fetched with the smallest box that covers them.
+struct KQMaps { CUtensorMap k[4], q[4], v[4]; };
+
 struct FParams {
     Params p;
-    int32_t tiles_per_unit;      // d_v / 128
+    int32_t heads_per_group;     // consecutive heads of one (layer, sequence) a CTA takes together
     long n_units;
 };
-
-// Byte offset of (row r, float e) inside the swizzled [K;Q] operand.
-__device__ __forceinline__ uint32_t bop_offset(int r, int e)
-{
-    const int c = e >> 5, w = (e >> 2) & 7;
-    return uint32_t(c * kBopChunkBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((w ^ (r & 7)) << 4) + ((e & 3) << 2));
-}
-
-template <int D>
-__device__ __forceinline__ void node_step(float (&ustk)[kMaxDepth], const float *cf, float Rv, float Gv, float vv,
-                                          float &u_out, float &o_out)
-{
-    // cf: cU[0..7] cO[0..7] cV cR cG
-    const float4 a0 = *reinterpret_cast<const float4 *>(cf + 0), a1 = *reinterpret_cast<const float4 *>(cf + 4);
-    const float4 b0 = *reinterpret_cast<const float4 *>(cf + 8), b1 = *reinterpret_cast<const float4 *>(cf + 12);
-    const float4 s = *reinterpret_cast<const float4 *>(cf + 16);
-    const float cU[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-    const float cO[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-    float u = fmaf(s.x, vv, s.y * Rv);
-    float o = s.z * Gv;
-#pragma unroll
-    for (int j = 0; j < D - 1; ++j) {
-        u = fmaf(cU[j], ustk[j], u);
-        o = fmaf(cO[j], ustk[j], o);
-    }
-    ustk[D - 1] = u;
-    o_out = fmaf(cO[D - 1], u, o);
-    u_out = u;
-}
 
 __device__ __forceinline__ int anc_byte(const int4 &meta, int j)
 {
     return int((j < 4 ? (uint32_t(meta.y) >> (8 * j)) : (uint32_t(meta.z) >> (8 * (j - 4)))) & 0xffu);
 }
 
+// kind::f16 with bf16 operands, fp32 accumulate, both operands K-major, M = 128 (Gram block)
+__device__ __forceinline__ uint32_t make_idesc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(kTileRows >> 4) << 24);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Units are taken in groups of HG consecutive heads of one (layer, sequence): group
+// G = blockIdx.x, += gridDim.x.  Inside a group the topology-dependent data (node count,
+// order, ancestors) is loaded once.  Sequences that failed validation or are empty are
+// skipped.  Every role walks the same list; unit number i of a CTA (unit_seq) uses
+// accumulator pair, coefficient buffer and epilogue group i & 1.
+struct Unit { int grp, hi, u, b, l, h, n, npad, base; };
+struct UnitWalk { int HG, gpl, n_groups, H, B, grid; const int32_t *seq_n; const int32_t *offs; };
+
+__device__ __forceinline__ bool load_group(const UnitWalk &w, int G, Unit &x)
+{
+    for (; G < w.n_groups; G += w.grid) {
+        const int lb = G / w.gpl;                        // (layer, sequence) pair
+        x.b = lb % w.B;
+        x.n = w.seq_n[x.b];
+        if (x.n > 0) {
+            x.grp = G;
+            x.hi = 0;
+            x.l = lb / w.B;
+            x.h = (G - lb * w.gpl) * w.HG;
+            x.u = lb * w.H + x.h;
+            x.npad = (x.n + 15) & ~15;
+            x.base = __ldg(w.offs + x.b);
+            return true;
+        }
+    }
+    x.n = 0; x.grp = w.n_groups;
+    return false;
+}
+__device__ __forceinline__ bool first_unit(const UnitWalk &w, Unit &x) { return load_group(w, int(blockIdx.x), x); }
+__device__ __forceinline__ bool next_unit(const UnitWalk &w, Unit &x)
+{
+    if (++x.hi < w.HG) { ++x.h; ++x.u; return true; }
+    return load_group(w, x.grp + w.grid, x);
+}
+
+// try once inline; fall into the bounded polling loop only if the barrier is not ready yet
+__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    return mbar_wait(bar, parity, abort_flag);
+}
+
+// One node of the forward substitution for TP value rows (one per tile of the unit),
+// branch-free.  The u of the nodes on the current depth-first path live in ustk[.][depth-1];
+// coefficients of levels that are not ancestors of this node are zero.
+//   cf[0..6] cU   cf[7] cV   cf[8..15] cO   cf[16] cR   cf[17] cG   cf[18] depth-1   cf[19] output offset
+template <int TP>
+__device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const float *cf, const float (&Rv)[TP],
+                                          const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
+                                          float (&o_out)[TP], int &off)
+{
+    const float4 a0 = *reinterpret_cast<const float4 *>(cf + 0), a1 = *reinterpret_cast<const float4 *>(cf + 4);
+    const float4 b0 = *reinterpret_cast<const float4 *>(cf + 8), b1 = *reinterpret_cast<const float4 *>(cf + 12);
+    const float4 s = *reinterpret_cast<const float4 *>(cf + 16);
+    const int d1 = __float_as_int(s.z);
+    off = __float_as_int(s.w);
+#pragma unroll
+    for (int t = 0; t < TP; ++t) {
+        float u0 = fmaf(a1.w, vv[t], s.x * Rv[t]);
+        float u1 = a0.y * ustk[t][1];
+        u0 = fmaf(a0.x, ustk[t][0], u0);
+        u1 = fmaf(a0.w, ustk[t][3], u1);
+        u0 = fmaf(a0.z, ustk[t][2], u0);
+        u1 = fmaf(a1.y, ustk[t][5], u1);
+        u0 = fmaf(a1.x, ustk[t][4], u0);
+        u0 = fmaf(a1.z, ustk[t][6], u0);
+        const float u = u0 + u1;
+#pragma unroll
+        for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        float o0 = fmaf(b0.x, ustk[t][0], s.y * Gv[t]);
+        float o1 = b0.y * ustk[t][1];
+        o0 = fmaf(b0.z, ustk[t][2], o0);
+        o1 = fmaf(b0.w, ustk[t][3], o1);
+        o0 = fmaf(b1.x, ustk[t][4], o0);
+        o1 = fmaf(b1.y, ustk[t][5], o1);
+        o0 = fmaf(b1.z, ustk[t][6], o0);
+        o1 = fmaf(b1.w, ustk[t][7], o1);
+        o_out[t] = o0 + o1;
+        u_out[t] = u;
+    }
+}
+
+// TP = value tiles per unit (d_v / 128): 1 or 2.
+template <int TP>
 __global__ void __launch_bounds__(kThreads, 1)
-verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
+verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
     extern __shared__ uint8_t smem_raw[];
     const Params &p = fp.p;
@@ -267,21 +394,21 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffMisc + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int TPU = fp.tiles_per_unit;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarFull + s), 1); mbar_init(bar(kBarEmpty + s), 1); }
         mbar_init(bar(kBarBReady), kPrepThreads);
         mbar_init(bar(kBarBFree), 1);
+        mbar_init(bar(kBarStageReady), 1);
         mbar_init(bar(kBarGramFull), 1);
+        mbar_init(bar(kBarGramDone), kPrepThreads);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarCoefReady + i), kPrepThreads);
-            mbar_init(bar(kBarCoefFree + i), 128 * TPU);
-            mbar_init(bar(kBarVReady + i), 128);
-            mbar_init(bar(kBarVFree + i), 128);
+            mbar_init(bar(kBarCoefFree + i), 128);
+            mbar_init(bar(kBarAccFull + i), 1);
+            mbar_init(bar(kBarPairFree + i), 128);
         }
-        for (int i = 0; i < kNumAcc; ++i) { mbar_init(bar(kBarAccFull + i), 1); mbar_init(bar(kBarAccFree + i), 128); }
         mbar_init(bar(kBarDrain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -291,37 +418,28 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Every role walks the same list of units: u = blockIdx.x, += gridDim.x, skipping
-    // sequences that failed validation or are empty.
-    struct Unit { long u; int b, l, h, n, npad, base; };
-    auto load_unit = [&](long u, Unit &x) {
-        x.u = u;
-        x.h = int(u % p.H); x.b = int((u / p.H) % p.B); x.l = int(u / (long(p.H) * p.B));
-        x.n = p.ws.seq_n[x.b];
-        x.npad = (x.n + 15) & ~15;
-        x.base = __ldg(p.node_offsets + x.b);
-    };
-    auto next_unit = [&](long from, Unit &x) {         // first valid unit at or after `from`; false at the end
-        for (long u = from; u < fp.n_units; u += gridDim.x) {
-            load_unit(u, x);
-            if (x.n > 0) return true;
-        }
-        x.u = fp.n_units; x.n = 0;
-        return false;
-    };
+    UnitWalk walk;
+    walk.HG = fp.heads_per_group; walk.gpl = p.H / fp.heads_per_group;
+    walk.n_groups = int(fp.n_units / fp.heads_per_group);
+    walk.H = p.H; walk.B = p.B; walk.grid = int(gridDim.x);
+    walk.seq_n = p.ws.seq_n; walk.offs = p.node_offsets;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
         uint32_t it = 0;
         Unit x;
         bool ok = true;
-        for (bool have = next_unit(blockIdx.x, x); have && ok; have = next_unit(x.u + gridDim.x, x)) {
-            for (int t = 0; t < TPU && ok; ++t) {
-                const int row = int(x.u * p.DV) + t * kTileRows;      // row in the [units*d_v, d_k] view of S0
+        PROF_DECL
+        for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
+            // the value rows of this unit's nodes are read by the epilogue with plain loads a
+            // couple of units from now: pull them into L2 meanwhile
+            if (lane == 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
+            for (int t = 0; t < TP && ok; ++t) {
+                const int row = x.u * p.DV + t * kTileRows;           // row in the [units*d_v, d_k] view of S0
                 for (int c = 0; c < kChunks; ++c, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
-                    if (!(ok = mbar_wait(bar(kBarEmpty + s), ph ^ 1, abort_flag))) break;
+                    if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
                     if (lane == 0) {
                         mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
                         tma_load_2d(sbase + kOffRing + s * kStageBytes, &s0_map, c * kChunkK, row, bar(kBarFull + s));
@@ -330,6 +448,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
                 }
             }
         }
+        PROF_STORE()
         // let copies still in flight land before the CTA's shared memory goes away
         if (*abort_flag) {
             const uint64_t t0 = global_timer_ns();
@@ -337,53 +456,67 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        uint32_t it = 0, unit_seq = 0, tile_seq = 0;
+        uint32_t it = 0, unit_seq = 0;
         Unit x;
         bool ok = true;
-        const uint32_t bop = sbase + kOffBop;
-        for (bool have = next_unit(blockIdx.x, x); have && ok; have = next_unit(x.u + gridDim.x, x), ++unit_seq) {
-            if (!(ok = mbar_wait(bar(kBarBReady), unit_seq & 1, abort_flag))) break;
+        const uint32_t bop = sbase + kOffBop, stage = sbase + kOffStage;
+        PROF_DECL
+        // Gram block of a unit: [K;Q] (128 rows) x K^T (npad columns) from the raw bf16 rows,
+        // parked in the unit's own accumulator columns until the state MMAs overwrite them.
+        auto issue_gram = [&](uint32_t seq, int npad) -> bool {
+            const int pr = seq & 1;
+            if (!WAIT(0, bar(kBarStageReady), seq & 1)) return false;
+            // the epilogue group must have released this pair of accumulators (unit seq - 2)
+            if (!WAIT(1, bar(kBarPairFree + pr), ((seq >> 1) & 1) ^ 1)) return false;
             tc_fence_after();
             if (lane == 0) {
-                // Gram block: [K;Q] (128 rows) x K^T (npad columns)
-                const uint32_t idg = make_idesc(x.npad);
-#pragma unroll 1
-                for (int c = 0; c < kChunks; ++c)
+                const uint32_t idg = make_idesc_bf16(npad);
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const uint64_t d = make_desc(bop + c * kBopChunkBytes + k * 32);
-                        mma_tf32(tmem_base + kGramCol, d, d, idg, (c | k) != 0);
+                        const uint64_t d = make_desc(stage + c * kStageChunkBytes + k * 32);
+                        mma_bf16(tmem_base + pr * kPairCols, d, d, idg, (c | k) != 0);
                     }
                 mma_commit(bar(kBarGramFull));
             }
             __syncwarp();
+            return true;
+        };
+        bool have = first_unit(walk, x);
+        if (have) ok = issue_gram(0, x.npad);
+        while (have && ok) {
+            const int pr = unit_seq & 1;
+            const uint32_t acc = tmem_base + pr * kPairCols;
+            if (!(ok = WAIT(2, bar(kBarBReady), unit_seq & 1))) break;
+            if (!(ok = WAIT(3, bar(kBarGramDone), unit_seq & 1))) break;
+            tc_fence_after();
             const uint32_t idm = make_idesc(2 * x.npad);
-            for (int t = 0; t < TPU && ok; ++t, ++tile_seq) {
-                const int a = tile_seq % kNumAcc;
-                const uint32_t aph = (tile_seq / kNumAcc) & 1;
-                if (!(ok = mbar_wait(bar(kBarAccFree + a), aph ^ 1, abort_flag))) break;
-                tc_fence_after();
+            for (int t = 0; t < TP && ok; ++t) {
                 for (int c = 0; c < kChunks; ++c, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
-                    if (!(ok = mbar_wait(bar(kBarFull + s), ph, abort_flag))) break;
+                    if (!(ok = WAIT(4, bar(kBarFull + s), ph))) break;
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t sa = sbase + kOffRing + s * kStageBytes;
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            mma_tf32(tmem_base + a * kAccCols, make_desc(sa + k * 32),
+                            mma_tf32(acc + t * kAccCols, make_desc(sa + k * 32),
                                      make_desc(bop + c * kBopChunkBytes + k * 32), idm, (c | k) != 0);
                         mma_commit(bar(kBarEmpty + s));
                     }
                     __syncwarp();
                 }
-                if (ok && lane == 0) mma_commit(bar(kBarAccFull + a));
-                __syncwarp();
             }
-            if (ok && lane == 0) mma_commit(bar(kBarBFree));
+            if (!ok) break;
+            if (lane == 0) { mma_commit(bar(kBarAccFull + pr)); mma_commit(bar(kBarBFree)); }
             __syncwarp();
+            ++unit_seq;
+            have = next_unit(walk, x);
+            if (have) ok = issue_gram(unit_seq, x.npad);
         }
+        PROF_STORE()
         // everything this warp issued must have completed before TMEM is released
         if (lane == 0) mma_commit(bar(kBarDrain));
         __syncwarp();
@@ -396,33 +529,56 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
         float *gram = reinterpret_cast<float *>(smem + kOffGram);
         float *alpha_s = reinterpret_cast<float *>(smem + kOffAlpha);
         float *beta_s = alpha_s + kMaxNodes;
-        const int sub = tid >> 4, e = (tid & 15) * 8;            // row within a group of 8, first of 8 floats
+        // Raw bf16 rows of [K;Q] of the NEXT unit are fetched by TMA, in node-index order, into a
+        // staging buffer laid out as a bf16 K-major 128-byte-swizzled operand: rows [0, npad) keys,
+        // [npad, 2 npad) queries.  The Gram MMA reads it directly; the conversion below gathers
+        // its rows in depth-first order into the fp32 operand of the state MMAs.
+        // This thread converts, for operand rows r = sub, sub + 8, ..., the 16-byte piece seg of
+        // the row (bf16 columns 8 seg .. 8 seg + 7).
+        const uint32_t stage = sbase + kOffStage;
+        const int sub = tid >> 4, seg = tid & 15;
+        // staging piece of node nd: chunk (seg >> 3) of 64 bf16, 16-byte slot (seg & 7) ^ (nd & 7)
+        const uint32_t stage_chunk = uint32_t((seg >> 3) * kStageChunkBytes);
+        // fp32 operand: floats 8 seg .. 8 seg + 7 -> chunk seg >> 2, 16-byte slots 2 (seg & 3), +1;
+        // r & 7 == sub for every handled row
+        const uint32_t bop_off0 = uint32_t((seg >> 2) * kBopChunkBytes + sub * 128 + (((2 * (seg & 3)) ^ sub) << 4));
+        const uint32_t bop_off1 = uint32_t((seg >> 2) * kBopChunkBytes + sub * 128 + (((2 * (seg & 3) + 1) ^ sub) << 4));
 
-        // raw bf16 rows of [K;Q] for the unit about to be written, fetched one unit ahead
-        uint4 raw[16];
         float my_alpha = 0.f, my_beta = 0.f;
+        unsigned long long node_lo = ~0ull, node_hi = ~0ull;   // node at the position of each handled row (0xff = none)
+        int topo_grp = -1;
+        int4 meta_nxt = make_int4(0, 0, 0, 0);
+        // start the TMA copies of unit x's rows (one thread), fetch alpha / beta and, when the
+        // sequence changes, the topology this thread needs
         auto prefetch = [&](const Unit &x) {
-            const int4 *anc = reinterpret_cast<const int4 *>(p.ws.anc) + x.base;
-            int node[16];
+            if (tid == 0) {
+                const int m = (x.npad >> 4) - 1;             // box height 16 (m + 1)
+                const int z = x.l * p.T + x.base;
+                mbar_arrive_expect_tx(bar(kBarStageReady), uint32_t(4 * x.npad * 128));
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int r = 8 * i + sub;
-                const int pos = r < x.npad ? r : r - x.npad;
-                node[i] = (r < 2 * x.npad && pos < x.n) ? ((__ldg(&anc[pos].x) >> 8) & 0xffff) : -1;
-            }
-            const int my_node = tid < x.n ? ((__ldg(&anc[tid].x) >> 8) & 0xffff) : -1;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int r = 8 * i + sub;
-                if (node[i] >= 0) {
-                    const long rec = (long(x.l) * p.T + x.base + node[i]) * p.H + x.h;
-                    raw[i] = __ldg(reinterpret_cast<const uint4 *>((r < x.npad ? p.k : p.q) + rec * kDK + e));
-                } else {
-                    raw[i] = make_uint4(0u, 0u, 0u, 0u);
+                for (int c = 0; c < 2; ++c) {
+                    tma_load_3d(stage + c * kStageChunkBytes, &kq.k[m], c * 64, x.h, z, bar(kBarStageReady));
+                    tma_load_3d(stage + c * kStageChunkBytes + x.npad * 128, &kq.q[m], c * 64, x.h, z, bar(kBarStageReady));
                 }
             }
-            if (my_node >= 0) {
-                const long rec = (long(x.l) * p.T + x.base + my_node) * p.H + x.h;
+            if (x.grp != topo_grp) {
+                topo_grp = x.grp;
+                node_lo = node_hi = 0ull;
+#pragma unroll 1
+                for (int i = 0; i < 16; ++i) {
+                    const int r = 8 * i + sub;
+                    const int pos = r < x.npad ? r : r - x.npad;
+                    const unsigned long long nd =
+                        (r < 2 * x.npad && pos < x.n) ? (unsigned long long)(__ldg(p.ws.plan + x.base + pos) & 0xff) : 0xffull;
+                    if (i < 8) node_lo |= nd << (8 * i);
+                    else node_hi |= nd << (8 * (i - 8));
+                }
+                const int node = row < x.npad ? row : row - x.npad;
+                meta_nxt = (row < 2 * x.npad && node < x.n)
+                               ? __ldg(reinterpret_cast<const int4 *>(p.ws.anc) + x.base + node) : make_int4(0, 0, 0, 0);
+            }
+            if (tid < x.n) {
+                const int rec = (x.l * p.T + x.base + tid) * p.H + x.h;
                 my_alpha = __ldg(p.alpha + rec);
                 my_beta = __ldg(p.beta + rec);
             }
@@ -431,25 +587,40 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
         uint32_t unit_seq = 0;
         Unit x, nx;
         bool ok = true;
-        bool have = next_unit(blockIdx.x, x);
+        bool have = first_unit(walk, x);
         if (have) prefetch(x);
+        int4 meta = meta_nxt;
+        unsigned long long cur_lo = node_lo, cur_hi = node_hi;
+        PROF_DECL
         for (; have && ok; ++unit_seq) {
             const int par = unit_seq & 1;
             // the previous unit's MMAs must be done reading the operand, and every prep thread
             // must be done reading alpha/beta of the previous unit
             if (unit_seq > 0) {
-                if (!(ok = mbar_wait(bar(kBarBFree), (unit_seq - 1) & 1, abort_flag))) break;
-                if (!(ok = mbar_wait(bar(kBarCoefReady + (par ^ 1)), ((unit_seq - 1) >> 1) & 1, abort_flag))) break;
+                if (!(ok = WAIT(0, bar(kBarBFree), (unit_seq - 1) & 1))) break;
+                if (!(ok = WAIT(1, bar(kBarCoefReady + (par ^ 1)), ((unit_seq - 1) >> 1) & 1))) break;
             }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int r = 8 * i + sub;
-                if (r < 2 * x.npad) {
-                    const uint4 w = raw[i];
-                    *reinterpret_cast<float4 *>(smem + kOffBop + bop_offset(r, e)) =
+            PROF_MARK()
+            // the staged rows of this unit have landed (the Gram MMA may still be reading them)
+            if (!(ok = WAIT(2, bar(kBarStageReady), unit_seq & 1))) break;
+            {
+                // bf16 -> fp32 (exact): operand row r (depth-first position) <- staged row of its node
+                const int iters = x.npad >> 2;               // 2 npad / 8
+                const int nk = x.npad >> 3;                  // rows [0, npad) keys, then queries
+                uint8_t *dst = smem + kOffBop;
+#pragma unroll 4
+                for (int i = 0; i < iters; ++i, dst += 1024) {
+                    const int nd = int(((i < 8 ? cur_lo : cur_hi) >> (8 * (i & 7))) & 0xffull);
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (nd != 0xff) {
+                        const int sr = i < nk ? nd : x.npad + nd;
+                        w = *reinterpret_cast<const uint4 *>(smem + kOffStage + stage_chunk + (sr >> 3) * 1024 + (sr & 7) * 128 +
+                                                            (((seg & 7) ^ (sr & 7)) << 4));
+                    }
+                    *reinterpret_cast<float4 *>(dst + bop_off0) =
                         make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u),
                                     __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u));
-                    *reinterpret_cast<float4 *>(smem + kOffBop + bop_offset(r, e + 4)) =
+                    *reinterpret_cast<float4 *>(dst + bop_off1) =
                         make_float4(__uint_as_float(w.z << 16), __uint_as_float(w.z & 0xffff0000u),
                                     __uint_as_float(w.w << 16), __uint_as_float(w.w & 0xffff0000u));
                 }
@@ -457,161 +628,215 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, FParams fp)
             if (tid < x.n) { alpha_s[tid] = my_alpha; beta_s[tid] = my_beta; }
             fence_proxy_async();
             mbar_arrive(bar(kBarBReady));
-            // start fetching the next unit's rows while this unit's Gram block is produced
-            const bool have_next = next_unit(x.u + gridDim.x, nx);
-            if (have_next) prefetch(nx);
-            // all prep threads have written alpha/beta (the operand barrier doubles as the prep barrier)
-            if (!(ok = mbar_wait(bar(kBarBReady), unit_seq & 1, abort_flag))) break;
-            // the coefficient buffer of this parity must have been released by the epilogue
-            if (unit_seq >= 2 && !(ok = mbar_wait(bar(kBarCoefFree + par), ((unit_seq >> 1) - 1) & 1, abort_flag))) break;
-            if (!(ok = mbar_wait(bar(kBarGramFull), unit_seq & 1, abort_flag))) break;
+            PROF_SEG(5)
+            if (!(ok = WAIT(3, bar(kBarGramFull), unit_seq & 1))) break;
             tc_fence_after();
+            PROF_MARK()
 
-            float *coef = reinterpret_cast<float *>(smem + kOffCoef) + par * kMaxNodes * kCoefStride;
-            const int4 *anc = reinterpret_cast<const int4 *>(p.ws.anc) + x.base;
+            // this thread's Gram row belongs to node `node` (keys: row, queries: row - npad)
             const bool is_k = row < x.npad;
-            const int pos = is_k ? row : row - x.npad;
-            const bool active = row < 2 * x.npad && pos < x.n;
-            int4 meta = make_int4(0, 0, 0, 0);
-            if (active) meta = __ldg(&anc[pos]);
+            const int node = is_k ? row : row - x.npad;
+            const bool in_rows = row < 2 * x.npad;
+            const bool active = in_rows && node < x.n;
             const int d = meta.x & 0xff;
-            float *cf = coef + pos * kCoefStride;
-            const float sgn = is_k ? -beta_s[active ? pos : 0] : p.scale;
-            for (int half = 0; half * kGramHalf < x.npad; ++half) {
-                // park this thread's Gram row (32 columns) in its private scratch column
+            const int pos = active ? ((meta.x >> 8) & 0xff) : node;       // padding rows: any unused record (n <= node < npad)
+            // ancestors by level (level d-1 is the node itself), their alpha, and this row's Gram entries
+            int anc_pos[kMaxDepth];
+            float anc_alpha[kMaxDepth], gsel[kMaxDepth];
 #pragma unroll
-                for (int c0 = 0; c0 < kGramHalf; c0 += 8) {
-                    float g[8];
-                    tmem_ld8(tmem_base + lane_addr + kGramCol + half * kGramHalf + c0, g);
+            for (int j = 0; j < kMaxDepth; ++j) anc_pos[j] = !active ? 0 : ((j < d - 1) ? anc_byte(meta, j) : node);
+
+            // park this thread's Gram row in its private scratch column (32 columns per pass),
+            // then pick the entries it needs
+            const uint32_t gaddr = tmem_base + par * kPairCols + lane_addr;
+#pragma unroll
+            for (int j = 0; j < kMaxDepth; ++j) gsel[j] = 0.f;
+#pragma unroll 1
+            for (int half = 0; half * kGramHalf < x.npad; ++half) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < kGramHalf; c0 += 16) {
+                    float g0[8], g1[8];
+                    tmem_ld8(gaddr + half * kGramHalf + c0, g0);
+                    tmem_ld8(gaddr + half * kGramHalf + c0 + 8, g1);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) gram[(c0 + i) * kTileRows + row] = g[i];
+                    for (int i = 0; i < 8; ++i) gram[(c0 + i) * kTileRows + row] = g0[i];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) gram[(c0 + 8 + i) * kTileRows + row] = g1[i];
                 }
-                if (active) {
-                    float ratio = alpha_s[pos];
-                    if (!is_k && (pos >> 5) == half) cf[8 + d - 1] = sgn * gram[(pos & 31) * kTileRows + row];
-                    for (int j = d - 2; j >= 0; --j) {
-                        const int a = anc_byte(meta, j);
-                        if ((a >> 5) == half) cf[(is_k ? 0 : 8) + j] = sgn * ratio * gram[(a & 31) * kTileRows + row];
-                        ratio *= alpha_s[a];
-                    }
-                    if (half == 0) {
-                        if (is_k) { cf[16] = -sgn; cf[17] = sgn * ratio; }          // cV = beta, cR = -beta gamma
-                        else { cf[18] = sgn * ratio; cf[19] = __int_as_float(meta.x); }   // cG = scale gamma, depth|node<<8
-                    }
-                }
+#pragma unroll
+                for (int j = 0; j < kMaxDepth; ++j)
+                    if ((anc_pos[j] >> 5) == half) gsel[j] = gram[(anc_pos[j] & 31) * kTileRows + row];
             }
             tc_fence_before();
+            mbar_arrive(bar(kBarGramDone));                  // the state MMAs may now overwrite these columns
+            PROF_SEG(7)
+            // The staging buffer may be refilled now: the Gram block of this unit is complete (the
+            // tensor core no longer reads the staged rows) and, once the operand barrier has
+            // completed, every prep thread has converted its rows (that barrier doubles as the
+            // prep-internal barrier for alpha / beta).
+            if (!(ok = WAIT(3, bar(kBarBReady), unit_seq & 1))) break;
+            nx = x;
+            const bool have_next = next_unit(walk, nx);
+            if (have_next) prefetch(nx);
+            PROF_SEG(6)
+#pragma unroll
+            for (int j = 0; j < kMaxDepth; ++j) anc_alpha[j] = alpha_s[anc_pos[j]];
+            const float my_a = alpha_s[active ? node : 0];
+            const float sgn = is_k ? -beta_s[active ? node : 0] : p.scale;
+            // the coefficient buffer of this parity must have been released by the epilogue
+            if (unit_seq >= 2 && !(ok = WAIT(4, bar(kBarCoefFree + par), ((unit_seq >> 1) - 1) & 1))) break;
+            // coefficient record of this row's node; levels that are not ancestors stay zero, rows
+            // past the last node (padding up to a multiple of 16) become no-op records
+            if (in_rows) {
+                float *cf = reinterpret_cast<float *>(smem + kOffCoef) + (par * kMaxNodes + pos) * kCoefStride;
+                float c[kMaxDepth];
+                float ratio = my_a;
+#pragma unroll
+                for (int j = kMaxDepth - 2; j >= 0; --j) {
+                    const bool is_anc = active && j < d - 1;
+                    c[j] = is_anc ? sgn * ratio * gsel[j] : 0.f;
+                    if (is_anc) ratio *= anc_alpha[j];
+                }
+                // after the loop ratio = gamma (product of alpha over the whole root path)
+                if (is_k) {
+                    c[7] = active ? -sgn : 0.f;                                       // cV = beta
+                    reinterpret_cast<float4 *>(cf)[0] = make_float4(c[0], c[1], c[2], c[3]);
+                    reinterpret_cast<float4 *>(cf)[1] = make_float4(c[4], c[5], c[6], c[7]);
+                    cf[16] = active ? sgn * ratio : 0.f;                              // cR = -beta gamma
+                } else {
+                    // level d-1 is the node itself: (q_t . k_t) with ratio 1
+                    c[7] = 0.f;
+#pragma unroll
+                    for (int j = 0; j < kMaxDepth; ++j)
+                        if (active && j == d - 1) c[j] = sgn * gsel[j];
+                    reinterpret_cast<float4 *>(cf)[2] = make_float4(c[0], c[1], c[2], c[3]);
+                    reinterpret_cast<float4 *>(cf)[3] = make_float4(c[4], c[5], c[6], c[7]);
+                    cf[17] = active ? sgn * ratio : 0.f;                              // cG = scale gamma
+                    cf[18] = __int_as_float(active ? d - 1 : -1);
+                    cf[19] = __int_as_float(active ? node * p.H * p.DV : 0);          // offset of the node's row
+                }
+            }
             mbar_arrive(bar(kBarCoefReady + par));
+            PROF_SEG(7)
             x = nx;
             have = have_next;
+            meta = meta_nxt;
+            cur_lo = node_lo; cur_hi = node_hi;
         }
+        PROF_STORE()
     } else {
         // ------------------------------------------------------------- epilogue groups
         const int grp = (warp - 6) >> 2;
-        const int gtid = threadIdx.x - (6 + 4 * grp) * 32;       // 0..127 within the group
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
-        const uint32_t vbuf = sbase + kOffVBuf + grp * kVBufBytes;
-        const unsigned short *vbuf_g = reinterpret_cast<const unsigned short *>(smem + kOffVBuf + grp * kVBufBytes);
+        const uint32_t acc = tmem_base + grp * kPairCols + lane_addr;
+        const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * kMaxNodes * kCoefStride;
+        const unsigned short *vraw = reinterpret_cast<const unsigned short *>(p.v);
 
-        struct Tile { Unit x; int t; uint32_t unit_seq, tile_seq; bool valid; };
-        // advance to the next tile owned by this group (tile_seq parity == grp)
-        auto advance = [&](Tile &tl, bool first) {
-            if (first) {
-                tl.valid = next_unit(blockIdx.x, tl.x);
-                tl.t = 0; tl.unit_seq = 0; tl.tile_seq = 0;
-                if (!tl.valid || int(tl.tile_seq & 1) == grp) return;
-            }
-            while (tl.valid) {
-                ++tl.tile_seq;
-                if (++tl.t == TPU) {
-                    tl.t = 0;
-                    ++tl.unit_seq;
-                    Unit nx;
-                    tl.valid = next_unit(tl.x.u + gridDim.x, nx);
-                    tl.x = nx;
-                }
-                if (tl.valid && int(tl.tile_seq & 1) == grp) return;
-            }
-        };
-        // stage the bf16 value tile [n][128 rows] of a tile into this group's buffer
-        auto stage_values = [&](const Tile &tl) {
-            if (tl.valid) {
-                const int4 *anc = reinterpret_cast<const int4 *>(p.ws.anc) + tl.x.base;
-                const long rec0 = (long(tl.x.l) * p.T + tl.x.base) * p.H + tl.x.h;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int idx = gtid + 128 * i, pos = idx >> 4, seg = idx & 15;
-                    if (pos < tl.x.n) {
-                        const int node = (__ldg(&anc[pos].x) >> 8) & 0xffff;
-                        const __nv_bfloat16 *src = p.v + (rec0 + long(node) * p.H) * p.DV + tl.t * kTileRows + seg * 8;
-                        cp_async_16(vbuf + pos * 256 + seg * 16, src);
-                    }
-                }
-            }
-            cp_async_arrive(bar(kBarVReady + grp));
-        };
-
-        Tile cur;
-        advance(cur, true);
-        stage_values(cur);
-        uint32_t my_seq = 0;                                     // tiles processed by this group
+        // this group's units: unit_seq == grp (mod 2)
+        Unit x;
+        bool have = first_unit(walk, x);
+        if (have && grp == 1) have = next_unit(walk, x);
+        uint32_t my_seq = 0;
         bool ok = true;
-        while (cur.valid && ok) {
-            const Unit &x = cur.x;
-            const int par = cur.unit_seq & 1;
-            const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + par * kMaxNodes * kCoefStride;
-            if (!(ok = mbar_wait(bar(kBarCoefReady + par), (cur.unit_seq >> 1) & 1, abort_flag))) break;
-            if (!(ok = mbar_wait(bar(kBarVReady + grp), my_seq & 1, abort_flag))) break;
-            const int a = cur.tile_seq % kNumAcc;
-            if (!(ok = mbar_wait(bar(kBarAccFull + a), (cur.tile_seq / kNumAcc) & 1, abort_flag))) break;
+        PROF_DECL
+        // Two register buffers (A, B) of kEpiChunk nodes each: TMEM columns R, G and the bf16
+        // value rows.  While one chunk is processed the loads of the next one are in flight.
+        float RA[TP][kEpiChunk], GA[TP][kEpiChunk], RB[TP][kEpiChunk], GB[TP][kEpiChunk];
+        unsigned short vA[kEpiChunk][TP], vB[kEpiChunk][TP];
+        // value rows of the first chunk of a unit, fetched ahead (node order from the plan)
+        auto fetch_first_values = [&](const Unit &y) {
+            const int rec0 = (y.l * p.T + y.base) * p.H + y.h;
+#pragma unroll
+            for (int i = 0; i < kEpiChunk; ++i) {
+                const int node = i < y.n ? (__ldg(p.ws.plan + y.base + i) & 0xffff) : 0;
+#pragma unroll
+                for (int t = 0; t < TP; ++t)
+                    vA[i][t] = __ldg(vraw + size_t(rec0 + node * p.H) * p.DV + t * kTileRows + row);
+            }
+        };
+        if (have) fetch_first_values(x);
+        while (have && ok) {
+            // look up this group's next unit now: its global loads overlap with this unit's work
+            Unit nx = x;
+            bool have_next = next_unit(walk, nx);
+            if (have_next) have_next = next_unit(walk, nx);
+            if (!(ok = WAIT(0, bar(kBarCoefReady + grp), my_seq & 1))) break;
+            if (!(ok = WAIT(2, bar(kBarAccFull + grp), my_seq & 1))) break;
             tc_fence_after();
-            const long rec0 = (long(x.l) * p.T + x.base) * p.H + x.h;          // record of node 0
-            const int vrow = cur.t * kTileRows + row;
-            float ustk[kMaxDepth];
+            const size_t rec0 = size_t((x.l * p.T + x.base) * p.H + x.h);        // record of node 0
+            const unsigned short *v_row = vraw + rec0 * p.DV + row;
+            float *o_row = p.o + rec0 * p.DV + row;
+            float *u_row = p.u != nullptr ? p.u + rec0 * p.DV + row : nullptr;
+            float ustk[TP][kMaxDepth];
 #pragma unroll
-            for (int j = 0; j < kMaxDepth; ++j) ustk[j] = 0.f;
-            for (int p0 = 0; p0 < x.n; p0 += 8) {
-                float Rv[8], Gv[8];
-                tmem_ld8(tmem_base + lane_addr + a * kAccCols + p0, Rv);
-                tmem_ld8(tmem_base + lane_addr + a * kAccCols + x.npad + p0, Gv);
-                tmem_ld_wait();
+            for (int t = 0; t < TP; ++t)
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (p0 + i < x.n) {
-                        const float *cf = coef + (p0 + i) * kCoefStride;
-                        const int meta = __float_as_int(cf[19]);
-                        const int d = meta & 0xff, node = (meta >> 8) & 0xffff;
-                        const float vv = __uint_as_float(uint32_t(vbuf_g[(p0 + i) * kTileRows + row]) << 16);
-                        float uo, oo;
-                        switch (d) {
-                        case 1: node_step<1>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 2: node_step<2>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 3: node_step<3>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 4: node_step<4>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 5: node_step<5>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 6: node_step<6>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        case 7: node_step<7>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        default: node_step<8>(ustk, cf, Rv[i], Gv[i], vv, uo, oo); break;
-                        }
-                        const long out = (rec0 + long(node) * p.H) * p.DV + vrow;
-                        p.o[out] = oo;
-                        if (p.u != nullptr) p.u[out] = uo;
+                for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = 0.f;
+            const int npad = x.npad, n = x.n;
+            auto load_tmem = [&](int p0, float (&R)[TP][kEpiChunk], float (&G)[TP][kEpiChunk]) {
+#pragma unroll
+                for (int t = 0; t < TP; ++t) {
+                    tmem_ld4(acc + t * kAccCols + p0, R[t]);
+                    tmem_ld4(acc + t * kAccCols + npad + p0, G[t]);
+                }
+            };
+            auto load_values = [&](int p0, unsigned short (&vv)[kEpiChunk][TP]) {
+#pragma unroll
+                for (int i = 0; i < kEpiChunk; ++i) {
+                    const int off = __float_as_int(coef[(p0 + i) * kCoefStride + 19]);   // p0 + i < npad
+#pragma unroll
+                    for (int t = 0; t < TP; ++t) vv[i][t] = __ldg(v_row + off + t * kTileRows);
+                }
+            };
+            auto process = [&](int p0, const float (&R)[TP][kEpiChunk], const float (&G)[TP][kEpiChunk],
+                               const unsigned short (&vv)[kEpiChunk][TP]) {
+#pragma unroll
+                for (int i = 0; i < kEpiChunk; ++i) {
+                    float r_[TP], g_[TP], v_[TP], uo[TP], oo[TP];
+                    int off;
+#pragma unroll
+                    for (int t = 0; t < TP; ++t) {
+                        r_[t] = R[t][i]; g_[t] = G[t][i];
+                        v_[t] = __uint_as_float(uint32_t(vv[i][t]) << 16);
                     }
+                    node_step<TP>(ustk, coef + (p0 + i) * kCoefStride, r_, g_, v_, uo, oo, off);
+                    if (p0 + i < n) {
+#pragma unroll
+                        for (int t = 0; t < TP; ++t) {
+                            o_row[off + t * kTileRows] = oo[t];
+                            if (u_row != nullptr) u_row[off + t * kTileRows] = uo[t];
+                        }
+                    }
+                }
+            };
+            // Software pipeline, one chunk deep: buffer A is processed while buffer B (the next
+            // chunk's TMEM columns and value rows) is in flight; B is then moved into A.
+            load_tmem(0, RA, GA);
+#pragma unroll 1
+            for (int p0 = 0; p0 < n; p0 += kEpiChunk) {
+                tmem_ld_wait();
+                const bool more = p0 + kEpiChunk < n;
+                if (more) { load_tmem(p0 + kEpiChunk, RB, GB); load_values(p0 + kEpiChunk, vB); }
+                process(p0, RA, GA, vA);
+                if (more) {
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int t = 0; t < TP; ++t)
+#pragma unroll
+                        for (int i = 0; i < kEpiChunk; ++i) { RA[t][i] = RB[t][i]; GA[t][i] = GB[t][i]; vA[i][t] = vB[i][t]; }
                 }
             }
             tc_fence_before();
-            mbar_arrive(bar(kBarAccFree + a));
-            mbar_arrive(bar(kBarCoefFree + par));
-            mbar_arrive(bar(kBarVFree + grp));
-            // next tile of this group: refill the value buffer once every thread has left it
-            advance(cur, false);
-            if (!(ok = mbar_wait(bar(kBarVFree + grp), my_seq & 1, abort_flag))) break;
+            mbar_arrive(bar(kBarPairFree + grp));
+            mbar_arrive(bar(kBarCoefFree + grp));
             ++my_seq;
-            stage_values(cur);
+            x = nx;
+            have = have_next;
+            if (have) fetch_first_values(x);
         }
-        asm volatile("cp.async.wait_all;" ::: "memory");
+        PROF_STORE()
     }
 
     tc_fence_before();
@@ -644,7 +869,8 @@ EncodeTiledFn encode_tiled_fn()
 
 bool factorized_supported(const speca_dims *d)
 {
-    return d->d_k == kDK && d->d_v % kTileRows == 0 && d->max_nodes <= kMaxNodes && d->max_depth <= kMaxDepth;
+    return d->d_k == kDK && (d->d_v == kTileRows || d->d_v == 2 * kTileRows) && d->max_nodes <= kMaxNodes &&
+           d->max_depth <= kMaxDepth;
 }
 
 int launch_verify_factorized(const Params &p, cudaStream_t st)
@@ -662,6 +888,30 @@ int launch_verify_factorized(const Params &p, cudaStream_t st)
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return int(cudaErrorInvalidValue);
 
+    KQMaps kq;
+    {
+        const cuuint64_t gd[3] = {cuuint64_t(kDK), cuuint64_t(p.H), cuuint64_t(p.L) * cuuint64_t(p.T)};
+        const cuuint64_t gs[2] = {cuuint64_t(kDK) * 2, cuuint64_t(p.H) * kDK * 2};
+        const cuuint32_t es[3] = {1, 1, 1};
+        for (int m = 0; m < 4; ++m) {
+            const cuuint32_t bx[3] = {64, 1, cuuint32_t(16 * (m + 1))};
+            CUresult r1 = encode(&kq.k[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16 *>(p.k), gd, gs, bx,
+                                 es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            CUresult r2 = encode(&kq.q[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16 *>(p.q), gd, gs, bx,
+                                 es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS) return int(cudaErrorInvalidValue);
+            const cuuint64_t vd[3] = {cuuint64_t(p.DV), cuuint64_t(p.H), cuuint64_t(p.L) * cuuint64_t(p.T)};
+            const cuuint64_t vs[2] = {cuuint64_t(p.DV) * 2, cuuint64_t(p.H) * p.DV * 2};
+            const cuuint32_t vb[3] = {cuuint32_t(p.DV), 1, cuuint32_t(16 * (m + 1))};
+            CUresult r3 = encode(&kq.v[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16 *>(p.v), vd, vs, vb,
+                                 es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r3 != CUDA_SUCCESS) return int(cudaErrorInvalidValue);
+        }
+    }
+
     static int sm_count = 0;
     if (sm_count == 0) {
         int dev = 0;
@@ -671,17 +921,22 @@ int launch_verify_factorized(const Params &p, cudaStream_t st)
     }
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(verify_factorized_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(verify_factorized_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(verify_factorized_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kSmemBytes);
         if (e != cudaSuccess) return int(e);
         attr_set = true;
     }
     FParams fp;
     fp.p = p;
-    fp.tiles_per_unit = p.DV / kTileRows;
     fp.n_units = n_units;
-    const int grid = int(n_units < sm_count ? n_units : sm_count);
-    verify_factorized_kernel<<<grid, kThreads, kSmemBytes, st>>>(map, fp);
+    fp.heads_per_group = (p.H % 4 == 0) ? 4 : (p.H % 2 == 0 ? 2 : 1);
+    const long n_groups = n_units / fp.heads_per_group;
+    const int grid = int(n_groups < sm_count ? n_groups : sm_count);
+    if (p.DV == kTileRows) verify_factorized_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+    else verify_factorized_kernel<2><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
     return int(cudaGetLastError());
 }
 

@@ -111,9 +111,9 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
         posn[i] = pos;
     }
     __syncthreads();
-    // Per position: depth, node index and the positions of the node's ancestors by depth
-    // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 8, which is
-    // all the factorised route accepts).
+    // Per node: depth, position in the processing order, and the node's ancestors by depth
+    // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 8, which is all
+    // the factorised route accepts).
     for (int i = tid; i < n; i += kPlanThreads) {
         int d = 0;
         for (int a = i; a >= 0; a = par[a]) ++d;
@@ -121,16 +121,16 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
         int j = d - 1;
         for (int a = par[i]; a >= 0; a = par[a]) {
             --j;
-            const uint32_t byte = uint32_t(posn[a]) & 0xffu;
+            const uint32_t byte = uint32_t(a) & 0xffu;
             if (j < 4) lo |= byte << (8 * j);
             else if (j < 8) hi |= byte << (8 * (j - 4));
         }
         int4 rec;
-        rec.x = d | (i << 8);
+        rec.x = d | (posn[i] << 8);
         rec.y = int(lo);
         rec.z = int(hi);
         rec.w = 0;
-        reinterpret_cast<int4 *>(ws.anc)[base + posn[i]] = rec;
+        reinterpret_cast<int4 *>(ws.anc)[base + i] = rec;
     }
     __syncthreads();
     if (tid == 0) {

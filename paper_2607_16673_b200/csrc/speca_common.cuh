@@ -12,13 +12,13 @@ namespace speca {
 
 // ---------------------------------------------------------------------------
 // Workspace layout (device scratch handed in by the caller).
-//   [0, 256)                     control words (work-queue counters)
-//   [256, 256 + 4*Bpad)          seq_n[b]: node count of sequence b, or -1 if the
+//   [0, 2048)                    control words (work-queue counters, optional profiling slots)
+//   [2048, 2048 + 4*Bpad)        seq_n[b]: node count of sequence b, or -1 if the
 //                                sequence failed validation and must be skipped
 //   then int32 arrays of Tpad words: plan[T], depth[T], anc[T][4]
 // Every region starts on a 256-byte boundary.
 // ---------------------------------------------------------------------------
-constexpr size_t kCtrlBytes = 256;
+constexpr size_t kCtrlBytes = 2048;
 constexpr int kNodeWords = 16;          // int32 words of scratch reserved per packed node
 
 __host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -28,7 +28,7 @@ struct Workspace {
     int32_t *seq_n;     // [B]
     int32_t *plan;      // [T]   packed schedule entries, in processing order per sequence
     int32_t *depth;     // [T]   depth computed from parent[]
-    int32_t *anc;       // [T][4] per processing position: depth | node << 8, ancestor positions (8 bytes), spare
+    int32_t *anc;       // [T][4] per node: depth | position << 8, ancestor node indices by level (8 bytes), spare
 };
 
 inline size_t workspace_bytes(int32_t batch, int32_t total_nodes)
