@@ -71,6 +71,7 @@ extern "C" {
 #define SPECA_ERR_RANGE        -4   /* a count is negative or too large                  */
 #define SPECA_ERR_CUDA         -5   /* the CUDA runtime reported an error at launch      */
 #define SPECA_ERR_WORKSPACE    -6   /* workspace NULL or smaller than required           */
+#define SPECA_ERR_TOO_LARGE    -7   /* problem exceeds the built-in scratch of a _noalloc entry point */
 
 /* bits of *status_word */
 #define SPECA_STATUS_BAD_PARENT   1   /* parent[i] < -1 or parent[i] >= i                          */
@@ -164,6 +165,43 @@ int speca_commit(const speca_dims *dims, float *S,
                  const int32_t *parent_or_null,
                  const int32_t *path_idx, const int32_t *path_len,
                  int32_t *status_word, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Variant of speca_verify_tree for callers that cannot provide scratch memory.
+ * (The paper has no counterpart: this is a property of the library, not of the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a serving loop
+ * whose memory pool is frozen after start-up, a plug-in that is handed tensors but no
+ * allocator, a latency-critical path where cudaMalloc (which synchronises the device)
+ * would stall every other stream.  Such a caller still owns the inputs and outputs, but
+ * has nowhere to take the verify workspace from.
+ *
+ * This entry point is speca_verify_tree with the workspace argument removed: the scratch
+ * (topology plan shared by all layers and heads) lives in a fixed array inside the library
+ * image, SPECA_NOALLOC_SCRATCH_BYTES per GPU that loads the library, held until the process
+ * exits.  It neither allocates nor frees device memory and calls nothing that does.
+ *
+ * Limits: dims->batch <= SPECA_NOALLOC_MAX_BATCH and total_nodes <= SPECA_NOALLOC_MAX_NODES,
+ * otherwise SPECA_ERR_TOO_LARGE and nothing is launched.
+ *
+ * The first call on each device looks up the device address of the array (a host-side
+ * query, no allocation); make that first call outside any stream capture.  Every call on
+ * a device uses the same array and finds in it whatever the previous call left; the
+ * kernels rewrite all of it they read, so nothing needs clearing by the caller -- but two
+ * calls whose kernels overlap on the GPU (different streams, no ordering between them)
+ * race on the array and must be serialised by the caller.
+ */
+#define SPECA_NOALLOC_MAX_BATCH   256
+#define SPECA_NOALLOC_MAX_NODES   16384
+#define SPECA_NOALLOC_SCRATCH_BYTES (2048 + 1024 + 16 * 65536)
+
+int speca_verify_tree_noalloc(const speca_dims *dims, const float *S0,
+                              const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                              const float *alpha, const float *beta,
+                              const int32_t *node_offsets, int32_t total_nodes,
+                              const int32_t *parent, const int32_t *depth_or_null,
+                              float *o, float *u_or_null,
+                              int32_t *status_word, void *stream);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,9 @@ STATUS_TOO_MANY, STATUS_TIMEOUT, STATUS_BAD_DEPTH = 16, 32, 64
 ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
-           "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit"]
+           "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
+           "speca_verify_tree_noalloc"]
+NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
 class SpecaError(RuntimeError):
@@ -75,10 +77,11 @@ def lib() -> ctypes.CDLL:
         L.speca_decode_step.argtypes = [dp] + [vp] * 8
         L.speca_verify_chain.argtypes = [dp] + [vp] * 7 + [i32, vp, vp, vp, sz, vp, vp]
         L.speca_verify_tree.argtypes = [dp] + [vp] * 7 + [i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.speca_verify_tree_noalloc.argtypes = [dp] + [vp] * 7 + [i32, vp, vp, vp, vp, vp, vp]
         L.speca_greedy_accept.argtypes = [i32, i32] + [vp] * 10
         L.speca_commit.argtypes = [dp] + [vp] * 6 + [i32] + [vp] * 5
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
-                     "speca_commit"):
+                     "speca_commit", "speca_verify_tree_noalloc"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -155,6 +158,21 @@ def verify_tree(dims: Dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes,
                                  _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(),
                                  _ptr(status, torch.int32, (1,), "status"), _stream())
     _check(rc, "speca_verify_tree")
+
+
+def verify_tree_noalloc(dims: Dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, parent, depth, o, u,
+                        status) -> None:
+    """speca_verify_tree without a workspace argument, for callers that may not allocate device
+    memory: the scratch is a fixed array inside the library (batch <= NOALLOC_MAX_BATCH,
+    total_nodes <= NOALLOC_MAX_NODES).  Calls on one device share that array, so calls that
+    could overlap on the GPU must be ordered by the caller."""
+    ins, outs = _verify_args(dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, o, u)
+    T = int(total_nodes)
+    d = dims.c()
+    rc = lib().speca_verify_tree_noalloc(ctypes.byref(d), *ins, T, _ptr(parent, torch.int32, (T,), "parent"),
+                                         _ptr(depth, torch.int32, (T,), "depth"), *outs,
+                                         _ptr(status, torch.int32, (1,), "status"), _stream())
+    _check(rc, "speca_verify_tree_noalloc")
 
 
 def greedy_accept(batch: int, max_depth: int, node_offsets, parent, draft_tok, target_tok, root_target_tok,

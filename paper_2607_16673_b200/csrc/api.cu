@@ -75,6 +75,29 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 
+// ---------------------------------------------------------------------------
+// Built-in scratch of speca_verify_tree_noalloc.  The array lives in the library image
+// on every device that loads it.  In host code its name is only a handle: the device
+// address has to be asked for, once per device, with that device current.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SPECA_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_noalloc_scratch_addr[kMaxDevices] = {};
+
+// Device address of the built-in scratch for the current device (nullptr on failure).
+void *noalloc_scratch_for_current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (g_noalloc_scratch_addr[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
+        g_noalloc_scratch_addr[dev] = ptr;
+    }
+    return g_noalloc_scratch_addr[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -91,6 +114,7 @@ const char *speca_strerror(int code)
     case SPECA_ERR_RANGE: return "a count is out of range";
     case SPECA_ERR_CUDA: return "CUDA launch error";
     case SPECA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SPECA_ERR_TOO_LARGE: return "batch or node count exceeds the built-in scratch of the _noalloc entry point";
     }
     return "unknown speca error code";
 }
@@ -136,6 +160,29 @@ int speca_verify_tree(const speca_dims *dims, const float *S0, const uint16_t *q
 {
     return verify_common(dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, parent, depth_or_null,
                          false, o, u_or_null, workspace, workspace_bytes, status_word, stream);
+}
+
+int speca_verify_tree_noalloc(const speca_dims *dims, const float *S0, const uint16_t *q, const uint16_t *k,
+                              const uint16_t *v, const float *alpha, const float *beta,
+                              const int32_t *node_offsets, int32_t total_nodes, const int32_t *parent,
+                              const int32_t *depth_or_null, float *o, float *u_or_null,
+                              int32_t *status_word, void *stream)
+{
+    if (dims == nullptr) return SPECA_ERR_NULL;
+    if (dims->batch > SPECA_NOALLOC_MAX_BATCH || total_nodes > SPECA_NOALLOC_MAX_NODES) return SPECA_ERR_TOO_LARGE;
+    static_assert(SPECA_NOALLOC_SCRATCH_BYTES >= kCtrlBytes + 4 * SPECA_NOALLOC_MAX_BATCH +
+                                                     size_t(kNodeWords) * 4 * SPECA_NOALLOC_MAX_NODES,
+                  "built-in scratch smaller than the workspace of the largest accepted problem");
+    // all argument checks first (they need no device); only then touch the CUDA runtime
+    void *scratch = nullptr;
+    if (total_nodes > 0 && dims->batch >= 1) {
+        scratch = noalloc_scratch_for_current_device();
+        if (scratch == nullptr) return SPECA_ERR_CUDA;
+    } else {
+        scratch = reinterpret_cast<void *>(uintptr_t(256));      // never dereferenced: nothing is launched
+    }
+    return verify_common(dims, S0, q, k, v, alpha, beta, node_offsets, total_nodes, parent, depth_or_null, false,
+                         o, u_or_null, scratch, SPECA_NOALLOC_SCRATCH_BYTES, status_word, stream);
 }
 
 int speca_greedy_accept(int32_t batch, int32_t max_depth, const int32_t *node_offsets,
