@@ -32,6 +32,8 @@
 // expiry the CTA raises SPECA_STATUS_TIMEOUT, drains and exits.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "speca_common.cuh"
 
 namespace speca {
@@ -435,14 +437,16 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             // couple of units from now: pull them into L2 meanwhile
             if (lane == 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
             for (int t = 0; t < TP && ok; ++t) {
-                const int row = x.u * p.DV + t * kTileRows;           // row in the [units*d_v, d_k] view of S0
+                // tile t of a unit holds its value rows t, t + TP, t + 2 TP, ... (interleaved tiles:
+                // an epilogue thread then owns TP ADJACENT value rows, one per tile)
+                const int row = x.u * kTileRows;                      // row-group in the [units*128][TP][d_k] view of S0
                 for (int c = 0; c < kChunks; ++c, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
                     if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
                     if (lane == 0) {
                         mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
-                        tma_load_2d(sbase + kOffRing + s * kStageBytes, &s0_map, c * kChunkK, row, bar(kBarFull + s));
+                        tma_load_3d(sbase + kOffRing + s * kStageBytes, &s0_map, c * kChunkK, t, row, bar(kBarFull + s));
                     }
                     __syncwarp();
                 }
@@ -732,7 +736,6 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
         const uint32_t acc = tmem_base + grp * kPairCols + lane_addr;
         const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * kMaxNodes * kCoefStride;
-        const unsigned short *vraw = reinterpret_cast<const unsigned short *>(p.v);
 
         // this group's units: unit_seq == grp (mod 2)
         Unit x;
@@ -744,16 +747,17 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         // Two register buffers (A, B) of kEpiChunk nodes each: TMEM columns R, G and the bf16
         // value rows.  While one chunk is processed the loads of the next one are in flight.
         float RA[TP][kEpiChunk], GA[TP][kEpiChunk], RB[TP][kEpiChunk], GB[TP][kEpiChunk];
-        unsigned short vA[kEpiChunk][TP], vB[kEpiChunk][TP];
+        // value rows: TP adjacent bf16 values per node, fetched with one load
+        using VPack = typename std::conditional<TP == 2, uint32_t, unsigned short>::type;
+        VPack vA[kEpiChunk], vB[kEpiChunk];
+        const VPack *vraw = reinterpret_cast<const VPack *>(p.v);
         // value rows of the first chunk of a unit, fetched ahead (node order from the plan)
         auto fetch_first_values = [&](const Unit &y) {
             const int rec0 = (y.l * p.T + y.base) * p.H + y.h;
 #pragma unroll
             for (int i = 0; i < kEpiChunk; ++i) {
                 const int node = i < y.n ? (__ldg(p.ws.plan + y.base + i) & 0xffff) : 0;
-#pragma unroll
-                for (int t = 0; t < TP; ++t)
-                    vA[i][t] = __ldg(vraw + size_t(rec0 + node * p.H) * p.DV + t * kTileRows + row);
+                vA[i] = __ldg(vraw + size_t(rec0 + node * p.H) * kTileRows + row);
             }
         };
         if (have) fetch_first_values(x);
@@ -766,9 +770,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (!(ok = WAIT(2, bar(kBarAccFull + grp), my_seq & 1))) break;
             tc_fence_after();
             const size_t rec0 = size_t((x.l * p.T + x.base) * p.H + x.h);        // record of node 0
-            const unsigned short *v_row = vraw + rec0 * p.DV + row;
-            float *o_row = p.o + rec0 * p.DV + row;
-            float *u_row = p.u != nullptr ? p.u + rec0 * p.DV + row : nullptr;
+            // this thread's TP adjacent value rows: row*TP .. row*TP + TP-1
+            const VPack *v_row = vraw + rec0 * kTileRows + row;
+            float *o_row = p.o + rec0 * p.DV + row * TP;
+            float *u_row = p.u != nullptr ? p.u + rec0 * p.DV + row * TP : nullptr;
             float ustk[TP][kMaxDepth];
 #pragma unroll
             for (int t = 0; t < TP; ++t)
@@ -782,16 +787,15 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     tmem_ld4(acc + t * kAccCols + npad + p0, G[t]);
                 }
             };
-            auto load_values = [&](int p0, unsigned short (&vv)[kEpiChunk][TP]) {
+            auto load_values = [&](int p0, VPack (&vv)[kEpiChunk]) {
 #pragma unroll
                 for (int i = 0; i < kEpiChunk; ++i) {
-                    const int off = __float_as_int(coef[(p0 + i) * kCoefStride + 19]);   // p0 + i < npad
-#pragma unroll
-                    for (int t = 0; t < TP; ++t) vv[i][t] = __ldg(v_row + off + t * kTileRows);
+                    const int off = __float_as_int(coef[(p0 + i) * kCoefStride + 19]);   // p0 + i < npad; in floats of o
+                    vv[i] = __ldg(v_row + off / TP);
                 }
             };
             auto process = [&](int p0, const float (&R)[TP][kEpiChunk], const float (&G)[TP][kEpiChunk],
-                               const unsigned short (&vv)[kEpiChunk][TP]) {
+                               const VPack (&vv)[kEpiChunk]) {
 #pragma unroll
                 for (int i = 0; i < kEpiChunk; ++i) {
                     float r_[TP], g_[TP], v_[TP], uo[TP], oo[TP];
@@ -799,14 +803,21 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                     for (int t = 0; t < TP; ++t) {
                         r_[t] = R[t][i]; g_[t] = G[t][i];
-                        v_[t] = __uint_as_float(uint32_t(vv[i][t]) << 16);
+                    }
+                    if (TP == 2) {
+                        v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
+                        v_[TP - 1] = __uint_as_float(uint32_t(vv[i]) & 0xffff0000u);
+                    } else {
+                        v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
                     }
                     node_step<TP>(ustk, coef + (p0 + i) * kCoefStride, r_, g_, v_, uo, oo, off);
                     if (p0 + i < n) {
-#pragma unroll
-                        for (int t = 0; t < TP; ++t) {
-                            o_row[off + t * kTileRows] = oo[t];
-                            if (u_row != nullptr) u_row[off + t * kTileRows] = uo[t];
+                        if (TP == 2) {
+                            *reinterpret_cast<float2 *>(o_row + off) = make_float2(oo[0], oo[TP - 1]);
+                            if (u_row != nullptr) *reinterpret_cast<float2 *>(u_row + off) = make_float2(uo[0], uo[TP - 1]);
+                        } else {
+                            o_row[off] = oo[0];
+                            if (u_row != nullptr) u_row[off] = uo[0];
                         }
                     }
                 }
@@ -825,7 +836,9 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                     for (int t = 0; t < TP; ++t)
 #pragma unroll
-                        for (int i = 0; i < kEpiChunk; ++i) { RA[t][i] = RB[t][i]; GA[t][i] = GB[t][i]; vA[i][t] = vB[i][t]; }
+                        for (int i = 0; i < kEpiChunk; ++i) { RA[t][i] = RB[t][i]; GA[t][i] = GB[t][i]; }
+#pragma unroll
+                    for (int i = 0; i < kEpiChunk; ++i) vA[i] = vB[i];
                 }
             }
             tc_fence_before();
@@ -879,11 +892,12 @@ int launch_verify_factorized(const Params &p, cudaStream_t st)
     if (encode == nullptr) return int(cudaErrorNotSupported);
     const long n_units = long(p.L) * p.B * p.H;
     CUtensorMap map;
-    const cuuint64_t gdim[2] = {cuuint64_t(kDK), cuuint64_t(n_units) * cuuint64_t(p.DV)};
-    const cuuint64_t gstride[1] = {cuuint64_t(kDK) * sizeof(float)};
-    const cuuint32_t box[2] = {kChunkK, kTileRows};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(p.S0), gdim, gstride, box, estr,
+    const int tiles = p.DV / kTileRows;
+    const cuuint64_t gdim[3] = {cuuint64_t(kDK), cuuint64_t(tiles), cuuint64_t(n_units) * kTileRows};
+    const cuuint64_t gstride[2] = {cuuint64_t(kDK) * sizeof(float), cuuint64_t(tiles) * kDK * sizeof(float)};
+    const cuuint32_t box[3] = {kChunkK, 1, kTileRows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(p.S0), gdim, gstride, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return int(cudaErrorInvalidValue);
