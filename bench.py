@@ -97,6 +97,25 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
+def rank_seed(base: int, rank: int, j: int = 0) -> int:
+    """Seed of input set j on a rank: every rank draws its own sequences (the batch is partitioned
+    over the ranks, a rank owns whole sequences), so seeds must differ across (rank, j)."""
+    return base + 97 * rank + j
+
+
+def reduce_over_ranks(dist, device, total_ms, t_verify, t_commit, tokens, vb, cb):
+    """Whole-job numbers: times are the MAX over ranks, processed units and bytes the SUM.
+    `dist` is torch.distributed (initialised) or None for a single process."""
+    if dist is None:
+        return total_ms, t_verify, t_commit, float(tokens), float(vb), float(cb)
+    import torch
+    tt = torch.tensor([total_ms, t_verify, t_commit], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    cnt = torch.tensor([tokens, vb, cb], device=device, dtype=torch.float64)
+    dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
+    return (float(tt[0]), float(tt[1]), float(tt[2]), float(cnt[0]), float(cnt[1]), float(cnt[2]))
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -170,11 +189,11 @@ def run_speca(args):
     stream = torch.cuda.current_stream()
 
     # --- inputs resident in HBM -------------------------------------------------
-    S = synth.device_state(1000 + rank, L, B, H, dk, dv, 0.02, dev)
+    S = synth.device_state(rank_seed(1000, rank), L, B, H, dk, dv, 0.02, dev)
     pool = []
     for j in range(POOL):
-        hi = host_round_inputs(args.workload, B, 5000 + 97 * rank + j)
-        q, k, v, al, be = synth.device_records(7000 + 97 * rank + j, L, hi["T"], H, dk, dv, dev)
+        hi = host_round_inputs(args.workload, B, rank_seed(5000, rank, j))
+        q, k, v, al, be = synth.device_records(rank_seed(7000, rank, j), L, hi["T"], H, dk, dv, dev)
         t = lambda a: torch.from_numpy(a).to(dev)
         pool.append(dict(hi, q=q, k=k, v=v, alpha=al, beta=be, d_offs=t(hi["node_offsets"]),
                          d_parent=t(hi["parent"]), d_depth=t(hi["depth"]), d_draft=t(hi["draft_tok"]),
@@ -245,15 +264,8 @@ def run_speca(args):
     t_accept = sum(e[1].elapsed_time(e[2]) for e in evs) / K
     t_commit = sum(e[2].elapsed_time(e[3]) for e in evs) / K
 
-    if world > 1:
-        tt = torch.tensor([total_ms, t_verify, t_commit], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, t_verify, t_commit = (float(x) for x in tt.tolist())
-        cnt = torch.tensor([tokens, vb, cb], device=dev, dtype=torch.float64)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        tokens_all = float(cnt[0]); vb_all = float(cnt[1]); cb_all = float(cnt[2])
-    else:
-        tokens_all, vb_all, cb_all = float(tokens), float(vb), float(cb)
+    total_ms, t_verify, t_commit, tokens_all, vb_all, cb_all = reduce_over_ranks(
+        dist if world > 1 else None, dev, total_ms, t_verify, t_commit, tokens, vb, cb)
 
     # --- decode-step baseline at the same batch (context) --------------------------
     q1, k1, v1, a1, b1 = synth.device_records(99, L, B, H, dk, dv, dev)
