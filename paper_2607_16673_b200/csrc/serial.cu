@@ -30,41 +30,51 @@ template <int G> __device__ __forceinline__ float group_sum(float x)
 }
 
 // 16 of a row's d_k values for this lane, from a bf16 vector in global memory.
-template <int G> __device__ __forceinline__ void load_vec(const __nv_bfloat16 *p, int g, float (&x)[16])
+// The 16 values a lane holds of a row are kept as 8 float2 so that the arithmetic can use the
+// packed two-wide fp32 instructions of sm_100 (each lane of a pair is an ordinary IEEE fp32 op).
+template <int G> __device__ __forceinline__ void load_vec(const __nv_bfloat16 *p, int g, float2 (&x)[8])
 {
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(p) + g + G * c);
-        x[4 * c + 0] = __uint_as_float(raw.x << 16);
-        x[4 * c + 1] = __uint_as_float(raw.x & 0xffff0000u);
-        x[4 * c + 2] = __uint_as_float(raw.y << 16);
-        x[4 * c + 3] = __uint_as_float(raw.y & 0xffff0000u);
+        x[2 * c + 0] = make_float2(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
+        x[2 * c + 1] = make_float2(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
     }
 }
 
-template <int G> __device__ __forceinline__ void load_row(const float *row, int g, float (&s)[16])
+template <int G> __device__ __forceinline__ void load_row(const float *row, int g, float2 (&s)[8])
 {
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         const float4 t = *(reinterpret_cast<const float4 *>(row) + g + G * c);
-        s[4 * c + 0] = t.x; s[4 * c + 1] = t.y; s[4 * c + 2] = t.z; s[4 * c + 3] = t.w;
+        s[2 * c + 0] = make_float2(t.x, t.y);
+        s[2 * c + 1] = make_float2(t.z, t.w);
     }
 }
 
-template <int G> __device__ __forceinline__ void store_row(float *row, int g, const float (&s)[16])
+template <int G> __device__ __forceinline__ void store_row(float *row, int g, const float2 (&s)[8])
 {
 #pragma unroll
     for (int c = 0; c < 4; ++c)
         *(reinterpret_cast<float4 *>(row) + g + G * c) =
-            make_float4(s[4 * c + 0], s[4 * c + 1], s[4 * c + 2], s[4 * c + 3]);
+            make_float4(s[2 * c + 0].x, s[2 * c + 0].y, s[2 * c + 1].x, s[2 * c + 1].y);
 }
 
-__device__ __forceinline__ float dot16(const float (&a)[16], const float (&b)[16])
+__device__ __forceinline__ float dot16(const float2 (&a)[8], const float2 (&b)[8])
 {
-    float acc0 = 0.f, acc1 = 0.f;
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int i = 0; i < 16; i += 2) { acc0 = fmaf(a[i], b[i], acc0); acc1 = fmaf(a[i + 1], b[i + 1], acc1); }
-    return acc0 + acc1;
+    for (int i = 0; i < 8; i += 2) { acc0 = __ffma2_rn(a[i], b[i], acc0); acc1 = __ffma2_rn(a[i + 1], b[i + 1], acc1); }
+    const float2 acc = __fadd2_rn(acc0, acc1);
+    return acc.x + acc.y;
+}
+
+// s <- alpha s + u k   (the rank-1 write of the rule)
+__device__ __forceinline__ void axpy16(float2 (&s)[8], const float2 (&k)[8], float alpha, float u)
+{
+    const float2 a2 = make_float2(alpha, alpha), u2 = make_float2(u, u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = __ffma2_rn(a2, s[i], __fmul2_rn(u2, k[i]));
 }
 
 __device__ __forceinline__ float bf16_to_float(const __nv_bfloat16 *p)
@@ -86,10 +96,10 @@ decode_kernel(Params p)
     const int lane = threadIdx.x & 31, g = lane % G, sub = lane / G;
 
     float *Su = p.S + unit * p.DV * DK;
-    float s[RS][16];
+    float2 s[RS][8];
 #pragma unroll
     for (int r = 0; r < RS; ++r) load_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
-    float kx[16], qx[16];
+    float2 kx[8], qx[8];
     load_vec<G>(p.k + unit * DK, g, kx);
     load_vec<G>(p.q + unit * DK, g, qx);
     const float alpha = __ldg(p.alpha + unit), beta = __ldg(p.beta + unit);
@@ -101,8 +111,7 @@ decode_kernel(Params p)
         const float sq = group_sum<G>(dot16(s[r], qx));
         const float vv = bf16_to_float(p.v + unit * p.DV + row);
         const float u = beta * (vv - alpha * sk);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
+        axpy16(s[r], kx, alpha, u);
         store_row<G>(Su + long(row) * DK, g, s[r]);
         if (g == 0) p.o[unit * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
     }
@@ -140,7 +149,7 @@ verify_serial_kernel(Params p)
     if (n <= 0) return;
 
     const float *S0u = p.S0 + unit * p.DV * DK;
-    float s[RS][16];
+    float2 s[RS][8];
 #pragma unroll
     for (int r = 0; r < RS; ++r) load_row<G>(S0u + long(row0 + r * RPS + sub) * DK, g, s[r]);
     float *my_slot = reinterpret_cast<float *>(slot_mem) + size_t(warp) * RS * RPS * DK;
@@ -165,7 +174,7 @@ verify_serial_kernel(Params p)
             }
         }
         const long rec = (long(l) * p.T + base + t) * p.H + h;
-        float kx[16], qx[16];
+        float2 kx[8], qx[8];
         load_vec<G>(p.k + rec * DK, g, kx);
         load_vec<G>(p.q + rec * DK, g, qx);
         const float alpha = __ldg(p.alpha + rec), beta = __ldg(p.beta + rec);
@@ -177,10 +186,7 @@ verify_serial_kernel(Params p)
             const float sq = group_sum<G>(dot16(s[r], qx));
             const float vv = bf16_to_float(p.v + rec * p.DV + row);
             const float u = beta * (vv - alpha * sk);
-            if (!leaf) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
-            }
+            if (!leaf) axpy16(s[r], kx, alpha, u);
             if (g == 0) {
                 p.o[rec * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
                 if (p.u != nullptr) p.u[rec * p.DV + row] = u;
@@ -198,7 +204,7 @@ verify_serial_kernel(Params p)
 // commit: advance S in place over the accepted factor records
 // ---------------------------------------------------------------------------
 template <int DK, int RS, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32)
+__global__ void __launch_bounds__(WARPS * 32, 2048 / (WARPS * 32) / 2)
 commit_kernel(Params p)
 {
     constexpr int G = Map<DK>::G, RPS = Map<DK>::RPS, ROWS = WARPS * RS * RPS;
@@ -208,46 +214,93 @@ commit_kernel(Params p)
     const int lane = threadIdx.x & 31, g = lane % G, sub = lane / G;
     const int row0 = (blockIdx.x % tiles) * ROWS + (threadIdx.x >> 5) * RS * RPS;
 
+    // path_len == 0: the sequence's state is neither read nor written
     const int len = __ldg(p.path_len + b);
-    if (len == 0) return;
     const int base = __ldg(p.node_offsets + b);
     const int n = __ldg(p.node_offsets + b + 1) - base;
-    // validate the whole path before touching the state (uniform over the CTA)
+    if (len == 0) return;
+
+    // Start streaming the state tile right away; the accepted path is validated in the
+    // shadow of these loads (one thread per path step), and nothing is stored if it is bad.
+    float *Su = p.S + unit * p.DV * DK;
+    float2 s[RS][8];
+    const bool len_ok = len > 0 && len <= p.max_depth;
+    if (len_ok) {
+#pragma unroll
+        for (int r = 0; r < RS; ++r) load_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
+    }
+    // The factor records of the whole accepted path (k rows, alpha, beta, the tile's v values)
+    // are staged in shared memory while the state tile is in flight, so that the token-by-token
+    // recurrence below never waits on global memory.
+    __shared__ int s_path[16];
+    __shared__ __align__(16) __nv_bfloat16 s_k[16][DK];
+    __shared__ float s_alpha[16], s_beta[16];
+    __shared__ __nv_bfloat16 s_v[16][ROWS];
     int fault = 0;
-    if (len < 0 || len > p.max_depth) fault = SPECA_STATUS_TOO_DEEP;
+    if (!len_ok) fault = SPECA_STATUS_TOO_DEEP;
     else if (base < 0 || n < 0 || base + n > p.T) fault = SPECA_STATUS_BAD_OFFSETS;
     else {
-        int prev = -1;
-        for (int d = 0; d < len; ++d) {
+        if (int(threadIdx.x) < len) {
+            const int d = threadIdx.x;
             const int t = __ldg(p.path_idx + b * p.max_depth + d);
-            if (t < 0 || t >= n) { fault = SPECA_STATUS_BAD_PATH; break; }
-            if (p.parent != nullptr && __ldg(p.parent + base + t) != prev) { fault = SPECA_STATUS_BAD_PATH; break; }
-            prev = t;
+            const int prev = d > 0 ? __ldg(p.path_idx + b * p.max_depth + d - 1) : -1;
+            if (t < 0 || t >= n) fault = SPECA_STATUS_BAD_PATH;
+            else if (p.parent != nullptr && __ldg(p.parent + base + t) != prev) fault = SPECA_STATUS_BAD_PATH;
+            s_path[d] = t;
+            if (!fault) {
+                const long rec = (long(l) * p.T + base + t) * p.H + h;
+                s_alpha[d] = __ldg(p.alpha + rec);
+                s_beta[d] = __ldg(p.beta + rec);
+            }
         }
+        constexpr int PIECES = DK / 8;                       // 16-byte pieces per k row
+        const int row_base = (blockIdx.x % tiles) * ROWS;
+        for (int idx = threadIdx.x; idx < len * PIECES; idx += WARPS * 32) {
+            const int d = idx / PIECES, piece = idx % PIECES;
+            const int t = __ldg(p.path_idx + b * p.max_depth + d);
+            if (t >= 0 && t < n) {
+                const long rec = (long(l) * p.T + base + t) * p.H + h;
+                const uint32_t dst = uint32_t(__cvta_generic_to_shared(&s_k[d][piece * 8]));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.k + rec * DK + piece * 8)
+                             : "memory");
+            }
+        }
+        for (int idx = threadIdx.x; idx < len * ROWS; idx += WARPS * 32) {
+            const int d = idx / ROWS, r = idx % ROWS;
+            const int t = __ldg(p.path_idx + b * p.max_depth + d);
+            if (t >= 0 && t < n) {
+                const long rec = (long(l) * p.T + base + t) * p.H + h;
+                s_v[d][r] = p.v[rec * p.DV + row_base + r];
+            }
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
     }
+    fault = __syncthreads_or(fault);
     if (fault) {
-        if (threadIdx.x == 0 && blockIdx.x % tiles == 0 && h == 0 && l == 0) atomicOr(p.status, fault);
+        // report one of the faults seen by the CTA (BAD_PATH is the only per-thread one)
+        if (threadIdx.x == 0 && blockIdx.x % tiles == 0 && h == 0 && l == 0)
+            atomicOr(p.status, !len_ok ? SPECA_STATUS_TOO_DEEP
+                                       : ((base < 0 || n < 0 || base + n > p.T) ? SPECA_STATUS_BAD_OFFSETS
+                                                                                : SPECA_STATUS_BAD_PATH));
         return;
     }
 
-    float *Su = p.S + unit * p.DV * DK;
-    float s[RS][16];
-#pragma unroll
-    for (int r = 0; r < RS; ++r) load_row<G>(Su + long(row0 + r * RPS + sub) * DK, g, s[r]);
+    const int tile_row = (threadIdx.x >> 5) * RS * RPS + sub;        // row inside the CTA's tile (row set 0)
     for (int d = 0; d < len; ++d) {
-        const int t = __ldg(p.path_idx + b * p.max_depth + d);
-        const long rec = (long(l) * p.T + base + t) * p.H + h;
-        float kx[16];
-        load_vec<G>(p.k + rec * DK, g, kx);
-        const float alpha = __ldg(p.alpha + rec), beta = __ldg(p.beta + rec);
+        float2 kx[8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint2 raw = *(reinterpret_cast<const uint2 *>(&s_k[d][0]) + g + G * c);
+            kx[2 * c + 0] = make_float2(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
+            kx[2 * c + 1] = make_float2(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+        }
+        const float alpha = s_alpha[d], beta = s_beta[d];
 #pragma unroll
         for (int r = 0; r < RS; ++r) {
-            const int row = row0 + r * RPS + sub;
             const float sk = group_sum<G>(dot16(s[r], kx));
-            const float vv = bf16_to_float(p.v + rec * p.DV + row);
+            const float vv = __bfloat162float(s_v[d][tile_row + r * RPS]);
             const float u = beta * (vv - alpha * sk);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) s[r][i] = fmaf(alpha, s[r][i], u * kx[i]);
+            axpy16(s[r], kx, alpha, u);
         }
     }
 #pragma unroll
