@@ -568,7 +568,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (x.grp != topo_grp) {
                 topo_grp = x.grp;
                 node_lo = node_hi = 0ull;
-#pragma unroll 1
+#pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const int r = 8 * i + sub;
                     const int pos = r < x.npad ? r : r - x.npad;
@@ -675,15 +675,9 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             tc_fence_before();
             mbar_arrive(bar(kBarGramDone));                  // the state MMAs may now overwrite these columns
             PROF_SEG(7)
-            // The staging buffer may be refilled now: the Gram block of this unit is complete (the
-            // tensor core no longer reads the staged rows) and, once the operand barrier has
-            // completed, every prep thread has converted its rows (that barrier doubles as the
-            // prep-internal barrier for alpha / beta).
+            // every prep thread has written alpha / beta and converted its rows (the operand barrier
+            // doubles as the prep-internal barrier)
             if (!(ok = WAIT(3, bar(kBarBReady), unit_seq & 1))) break;
-            nx = x;
-            const bool have_next = next_unit(walk, nx);
-            if (have_next) prefetch(nx);
-            PROF_SEG(6)
 #pragma unroll
             for (int j = 0; j < kMaxDepth; ++j) anc_alpha[j] = alpha_s[anc_pos[j]];
             const float my_a = alpha_s[active ? node : 0];
@@ -723,6 +717,12 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             }
             mbar_arrive(bar(kBarCoefReady + par));
             PROF_SEG(7)
+            // The staging buffer may be refilled now: the Gram block of this unit is complete (the
+            // tensor core no longer reads the staged rows) and every prep thread has converted its rows.
+            nx = x;
+            const bool have_next = next_unit(walk, nx);
+            if (have_next) prefetch(nx);
+            PROF_SEG(6)
             x = nx;
             have = have_next;
             meta = meta_nxt;
