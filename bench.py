@@ -44,7 +44,7 @@ POOL = 3            # independent draft inputs rotated over the steps ("fresh dr
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
@@ -117,24 +117,41 @@ def reduce_over_ranks(dist, device, total_ms, t_verify, t_commit, tokens, vb, cb
 
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """Samples SM clocks and throttle reasons with nvidia-smi while the benchmark runs.  It is
+    started before the warm-up (nvidia-smi needs a moment to come up); `mark()` brackets the timed
+    region and only samples inside the marks are summarised (all samples if none fell inside)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.proc = None
+        self.marks = []
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+            time.sleep(0.5)
         except Exception:
             self.proc = None
+
+    def mark(self):
+        self.marks.append(time.time())
+
+    @staticmethod
+    def _ts(text: str):
+        import datetime
+        try:
+            return datetime.datetime.strptime(text.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -142,24 +159,32 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.tmp.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
+                rows.append((self._ts(parts[0]), float(parts[1]), float(parts[2]),
+                             [nm for nm, val in zip(names, parts[4:8]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
         self.tmp.close()
         os.unlink(self.tmp.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        inside = rows
+        if len(self.marks) >= 2:
+            lo, hi = self.marks[0] - 0.02, self.marks[-1] + 0.02
+            sel = [r for r in rows if r[0] is not None and lo <= r[0] <= hi]
+            if sel:
+                inside = sel
+                out["window"] = "timed region"
+            else:
+                out["window"] = "whole run (no sample fell inside the timed region)"
+        if inside:
+            out.update(sm_mhz=float(np.median([r[1] for r in inside])), sm_max_mhz=float(max(r[2] for r in inside)),
+                       samples=len(inside))
+            out["reasons"] = sorted({nm for r in inside for nm in r[3]})
         return out
 
 
@@ -235,21 +260,23 @@ def run_speca(args):
         torch.cuda.synchronize()
         p["path_len"] = path_len.cpu().numpy().copy()
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for w in range(args.warmup):
         step(pool[w % POOL])
     barrier()
 
     K = args.steps
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     barrier()
+    if sampler: sampler.mark()
     t_start.record(stream)
     for i in range(K):
         step(pool[(args.warmup + i) % POOL], evs[i])
     t_end.record(stream)
     barrier()
+    if sampler: sampler.mark()
     clocks = sampler.stop() if sampler else None
     total_ms = t_start.elapsed_time(t_end)
     assert int(status.item()) == 0, f"device status word {int(status.item())}"
