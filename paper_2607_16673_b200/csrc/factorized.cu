@@ -385,11 +385,16 @@ template <int TP>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
-    extern __shared__ uint8_t smem_raw[];
+    // The swizzled operand regions need 1024-byte alignment.  The array is declared with that
+    // alignment and used directly, so every access below stays a shared-memory access for the
+    // compiler (address space known, no aliasing with the global output pointers).
+    extern __shared__ __align__(1024) uint8_t smem[];
     const Params &p = fp.p;
-    // 1024-byte alignment for the swizzled operand regions
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {                                 // never expected; refuse to run rather than corrupt
+        if (threadIdx.x == 0) atomicOr(p.status, SPECA_STATUS_TIMEOUT);
+        return;
+    }
     const uint32_t bars = sbase + kOffBars;
     auto bar = [&](int i) { return bars + 8u * uint32_t(i); };
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffMisc);
