@@ -341,7 +341,7 @@ def run_speca(args):
                    "input_pool": POOL, "l2": "inputs larger than L2 (state 6.4 GB, records 1.8 GB per round at full size)",
                    "route": args.route, "parallelism": f"dp{world} (sequences partitioned, no collective)"},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get(dom),
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get(dom) if args.workload == "cfg5" and not args.layers and not args.batch else None,
                      "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms},
         "kernels": {"verify_ms": t_verify, "accept_ms": t_accept, "commit_ms": t_commit,
                     "verify_gbs": vb / K / (t_verify * 1e-3) / 1e9, "commit_gbs": cb / K / (t_commit * 1e-3) / 1e9,
@@ -364,7 +364,7 @@ def run_speca(args):
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant
 # kernels from the ncu captures summarised under profiles/; None until captured.
-NCU_TRAFFIC = {"verify": None, "commit": None}
+NCU_TRAFFIC = {"verify": 12 * 835.9e6, "commit": 12 * 716.9e6}     # 2-layer captures x 12 (traffic is proportional to units)
 
 
 def run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream):
