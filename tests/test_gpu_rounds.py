@@ -100,3 +100,13 @@ def test_cfg5_shaped_16_rounds(route, tol):
 @pytest.mark.parametrize("route,tol", [(speca.ROUTE_SERIAL, TOL_FP32 * 4), (speca.ROUTE_AUTO, TOL)])
 def test_cfg4_shaped_rounds(route, tol):
     run_rounds("cfg4", 3, 32, 4, route, tol)
+
+
+def test_cfg5_full_size_sampled():
+    """The benchmark's own launch configuration (24 layers x 128 sequences x 16 heads, 6.4 GB of state),
+    two rounds, checked on sampled units."""
+    run_rounds("cfg5", 24, 128, 2, speca.ROUTE_AUTO, TOL, n_sample=32, seed=91)
+
+
+def test_cfg4_full_size_sampled():
+    run_rounds("cfg4", 24, 32, 2, speca.ROUTE_AUTO, TOL, n_sample=32, seed=92)
