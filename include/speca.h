@@ -166,6 +166,50 @@ int speca_commit(const speca_dims *dims, float *S,
                  const int32_t *path_idx, const int32_t *path_len,
                  int32_t *status_word, void *stream);
 
+/* Fused commit-and-verify: the delayed state update of Section 5.2 ("update fused into
+ * the next verification", Eq. 3 applied while the state tile is on chip).  Equivalent to
+ *     speca_commit(S, previous draft's records, path_idx, path_len)   followed by
+ *     speca_verify_tree(S, new draft)
+ * but the state crosses HBM twice (one read, one write) instead of three times.
+ *
+ * Pending commit: k_prev, v_prev, alpha_prev, beta_prev are the previous draft's records
+ * (layouts as in speca_verify_tree, packed by node_offsets_prev, total_nodes_prev nodes),
+ * path_idx / path_len its accepted paths as written by speca_greedy_accept, and
+ * u_prev_or_null the `u` the previous verification wrote for that draft ([L,Tp,H,d_v]).
+ * Each path must be a root path of the previous draft's tree (a node's u embeds its
+ * ancestors, so u of nodes that do not form such a path cannot be combined); pass
+ * parent_prev_or_null to have that checked.  A
+ * sequence with an invalid path gets STATUS_BAD_PATH / TOO_DEEP, its state is not
+ * advanced, and its new draft is verified from the state as it stands (exactly what the
+ * two separate calls do).  A sequence whose new tree is empty or rejected still gets its
+ * commit.  total_nodes_prev == 0 means nothing is pending (plain verification, S is not
+ * written); total_nodes == 0 means nothing to verify (plain commit).
+ *
+ * New draft and outputs: as speca_verify_tree, except that S is read and written.  Pass
+ * u_or_null to be able to fuse the next round; it must not be the buffer u_prev_or_null
+ * points to, and o / u must not alias any input.
+ *
+ * The single-pass kernel runs when the tensor-core route applies (d_k = 128, d_v in
+ * {128, 256}, max_nodes <= 64, max_depth <= 8, route != SERIAL) and u_prev_or_null is
+ * given: the pending update is then S <- gamma_A S + sum_i (gamma_A / gamma_i) u_i k_i^T,
+ * which needs only u, k and alpha of the accepted nodes (v_prev and beta_prev are not
+ * read).  Otherwise the commit and verify kernels are launched back to back on `stream`
+ * with the same results.  workspace_bytes must be at least speca_workspace_bytes(). */
+int speca_commit_verify_tree(const speca_dims *dims, float *S,
+                             const uint16_t *k_prev, const uint16_t *v_prev,
+                             const float *alpha_prev, const float *beta_prev,
+                             const float *u_prev_or_null,
+                             const int32_t *node_offsets_prev, int32_t total_nodes_prev,
+                             const int32_t *parent_prev_or_null,
+                             const int32_t *path_idx, const int32_t *path_len,
+                             const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                             const float *alpha, const float *beta,
+                             const int32_t *node_offsets, int32_t total_nodes,
+                             const int32_t *parent, const int32_t *depth_or_null,
+                             float *o, float *u_or_null,
+                             void *workspace, size_t workspace_bytes,
+                             int32_t *status_word, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Variant of speca_verify_tree for callers that cannot provide scratch memory.
  * (The paper has no counterpart: this is a property of the library, not of the method.)
@@ -193,7 +237,7 @@ int speca_commit(const speca_dims *dims, float *S,
  */
 #define SPECA_NOALLOC_MAX_BATCH   256
 #define SPECA_NOALLOC_MAX_NODES   16384
-#define SPECA_NOALLOC_SCRATCH_BYTES (2048 + 1024 + 16 * 65536)
+#define SPECA_NOALLOC_SCRATCH_BYTES (2048 + 1024 + 16 * 65536 + 12288)
 
 int speca_verify_tree_noalloc(const speca_dims *dims, const float *S0,
                               const uint16_t *q, const uint16_t *k, const uint16_t *v,

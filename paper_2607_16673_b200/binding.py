@@ -25,7 +25,7 @@ ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
-           "speca_verify_tree_noalloc"]
+           "speca_verify_tree_noalloc", "speca_commit_verify_tree"]
 NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
@@ -80,8 +80,10 @@ def lib() -> ctypes.CDLL:
         L.speca_verify_tree_noalloc.argtypes = [dp] + [vp] * 7 + [i32, vp, vp, vp, vp, vp, vp]
         L.speca_greedy_accept.argtypes = [i32, i32] + [vp] * 10
         L.speca_commit.argtypes = [dp] + [vp] * 6 + [i32] + [vp] * 5
+        L.speca_commit_verify_tree.argtypes = ([dp] + [vp] * 7 + [i32] + [vp] * 3 + [vp] * 6 + [i32] + [vp] * 5 +
+                                               [sz, vp, vp])
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
-                     "speca_commit", "speca_verify_tree_noalloc"):
+                     "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -200,3 +202,37 @@ def commit(dims: Dims, S, k, v, alpha, beta, node_offsets, total_nodes, parent, 
         _ptr(path_idx, i32, (B, dims.max_depth), "path_idx"), _ptr(path_len, i32, (B,), "path_len"),
         _ptr(status, i32, (1,), "status"), _stream())
     _check(rc, "speca_commit")
+
+
+def commit_verify_tree(dims: Dims, S, prev, path_idx, path_len, q, k, v, alpha, beta, node_offsets, total_nodes,
+                       parent, depth, o, u, workspace, status) -> None:
+    """speca_commit_verify_tree: commit the previous draft's accepted paths into S and verify the
+    new draft from the committed state.  ``prev`` is None (nothing pending) or a dict with the
+    previous draft's ``k, v, alpha, beta`` records, ``u`` (what its verification wrote, or None),
+    ``node_offsets``, ``total_nodes`` and ``parent`` (or None)."""
+    L, B, H, dk, dv, T = dims.n_layers, dims.batch, dims.heads, dims.d_k, dims.d_v, int(total_nodes)
+    i32 = torch.int32
+    if prev is None:
+        pargs = [None] * 5 + [None, 0, None]
+        Tp = 0
+    else:
+        Tp = int(prev["total_nodes"])
+        pargs = [_ptr(prev["k"], torch.bfloat16, (L, Tp, H, dk), "k_prev"),
+                 _ptr(prev["v"], torch.bfloat16, (L, Tp, H, dv), "v_prev"),
+                 _ptr(prev["alpha"], torch.float32, (L, Tp, H), "alpha_prev"),
+                 _ptr(prev["beta"], torch.float32, (L, Tp, H), "beta_prev"),
+                 _ptr(prev.get("u"), torch.float32, (L, Tp, H, dv), "u_prev"),
+                 _ptr(prev["node_offsets"], i32, (B + 1,), "node_offsets_prev"), Tp,
+                 _ptr(prev.get("parent"), i32, (Tp,), "parent_prev")]
+    d = dims.c()
+    rc = lib().speca_commit_verify_tree(
+        ctypes.byref(d), _ptr(S, torch.float32, (L, B, H, dv, dk), "S"), *pargs,
+        _ptr(path_idx, i32, (B, dims.max_depth), "path_idx"), _ptr(path_len, i32, (B,), "path_len"),
+        _ptr(q, torch.bfloat16, (L, T, H, dk), "q"), _ptr(k, torch.bfloat16, (L, T, H, dk), "k"),
+        _ptr(v, torch.bfloat16, (L, T, H, dv), "v"), _ptr(alpha, torch.float32, (L, T, H), "alpha"),
+        _ptr(beta, torch.float32, (L, T, H), "beta"), _ptr(node_offsets, i32, (B + 1,), "node_offsets"), T,
+        _ptr(parent, i32, (T,), "parent"), _ptr(depth, i32, (T,), "depth"),
+        _ptr(o, torch.float32, (L, T, H, dv), "o"), _ptr(u, torch.float32, (L, T, H, dv), "u"),
+        _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(),
+        _ptr(status, i32, (1,), "status"), _stream())
+    _check(rc, "speca_commit_verify_tree")

@@ -71,7 +71,7 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
         rc = cuda_rc(launch_plan(p, st));
         if (rc != SPECA_OK) return rc;
     }
-    if (factorize) return cuda_rc(launch_verify_factorized(p, st));
+    if (factorize) return cuda_rc(launch_verify_factorized(p, false, st));
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 
@@ -171,7 +171,8 @@ int speca_verify_tree_noalloc(const speca_dims *dims, const float *S0, const uin
     if (dims == nullptr) return SPECA_ERR_NULL;
     if (dims->batch > SPECA_NOALLOC_MAX_BATCH || total_nodes > SPECA_NOALLOC_MAX_NODES) return SPECA_ERR_TOO_LARGE;
     static_assert(SPECA_NOALLOC_SCRATCH_BYTES >= kCtrlBytes + 4 * SPECA_NOALLOC_MAX_BATCH +
-                                                     size_t(kNodeWords) * 4 * SPECA_NOALLOC_MAX_NODES,
+                                                     size_t(kNodeWords) * 4 * SPECA_NOALLOC_MAX_NODES +
+                                                     size_t(kPendWords) * 4 * SPECA_NOALLOC_MAX_BATCH,
                   "built-in scratch smaller than the workspace of the largest accepted problem");
     // all argument checks first (they need no device); only then touch the CUDA runtime
     void *scratch = nullptr;
@@ -220,6 +221,74 @@ int speca_commit(const speca_dims *dims, float *S, const uint16_t *k, const uint
     p.node_offsets = node_offsets; p.parent = parent_or_null;
     p.path_idx = path_idx; p.path_len = path_len; p.status = status_word;
     return cuda_rc(launch_commit(p, dims->d_k, static_cast<cudaStream_t>(stream)));
+}
+
+int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k_prev, const uint16_t *v_prev,
+                             const float *alpha_prev, const float *beta_prev, const float *u_prev_or_null,
+                             const int32_t *node_offsets_prev, int32_t total_nodes_prev,
+                             const int32_t *parent_prev_or_null, const int32_t *path_idx, const int32_t *path_len,
+                             const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *alpha,
+                             const float *beta, const int32_t *node_offsets, int32_t total_nodes,
+                             const int32_t *parent, const int32_t *depth_or_null, float *o, float *u_or_null,
+                             void *workspace, size_t workspace_bytes, int32_t *status_word, void *stream)
+{
+    int rc = check_dims(dims);
+    if (rc != SPECA_OK) return rc;
+    if (!S || !status_word) return SPECA_ERR_NULL;
+    if (total_nodes_prev < 0 || total_nodes < 0) return SPECA_ERR_RANGE;
+    const bool have_commit = total_nodes_prev > 0;
+    if (have_commit && (!k_prev || !v_prev || !alpha_prev || !beta_prev || !node_offsets_prev || !path_idx || !path_len))
+        return SPECA_ERR_NULL;
+    if (have_commit && (misaligned(k_prev) || misaligned(v_prev) || misaligned(alpha_prev) || misaligned(beta_prev) ||
+                        (u_prev_or_null && misaligned(u_prev_or_null))))
+        return SPECA_ERR_ALIGN;
+    if (total_nodes > 0 && workspace_bytes < speca::workspace_bytes(dims->batch, total_nodes))
+        return SPECA_ERR_WORKSPACE;
+
+    // One pass over the state when the tensor-core route applies and the previous verification
+    // left its u; otherwise the two kernels run back to back on the stream (same results).
+    const bool one_pass = have_commit && total_nodes > 0 && u_prev_or_null != nullptr && factorized_supported(dims) &&
+                          dims->route != SPECA_ROUTE_SERIAL;
+    if (!one_pass) {
+        if (have_commit) {
+            rc = speca_commit(dims, S, k_prev, v_prev, alpha_prev, beta_prev, node_offsets_prev, total_nodes_prev,
+                              parent_prev_or_null, path_idx, path_len, status_word, stream);
+            if (rc != SPECA_OK) return rc;
+        }
+        if (total_nodes == 0) return SPECA_OK;
+        return verify_common(dims, S, q, k, v, alpha, beta, node_offsets, total_nodes, parent, depth_or_null, false, o,
+                             u_or_null, workspace, workspace_bytes, status_word, stream);
+    }
+
+    if (!q || !k || !v || !alpha || !beta || !node_offsets || !parent || !o) return SPECA_ERR_NULL;
+    if (1LL * total_nodes > 1LL * dims->batch * dims->max_nodes) return SPECA_ERR_RANGE;
+    if (misaligned(S) || misaligned(q) || misaligned(k) || misaligned(v) || misaligned(alpha) || misaligned(beta) ||
+        misaligned(o) || (u_or_null && misaligned(u_or_null)) || misaligned(node_offsets) || misaligned(parent) ||
+        (depth_or_null && misaligned(depth_or_null)))
+        return SPECA_ERR_ALIGN;
+    if (!workspace || misaligned(workspace)) return SPECA_ERR_WORKSPACE;
+    if (u_or_null != nullptr && u_or_null == u_prev_or_null) return SPECA_ERR_RANGE;     // read and written in one pass
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Params p = base_params(dims, total_nodes);
+    p.S = S; p.S0 = S;
+    p.q = reinterpret_cast<const __nv_bfloat16 *>(q);
+    p.k = reinterpret_cast<const __nv_bfloat16 *>(k);
+    p.v = reinterpret_cast<const __nv_bfloat16 *>(v);
+    p.alpha = alpha; p.beta = beta; p.o = o; p.u = u_or_null;
+    p.node_offsets = node_offsets; p.parent = parent; p.depth_in = depth_or_null;
+    p.path_idx = path_idx; p.path_len = path_len;
+    p.pk = reinterpret_cast<const __nv_bfloat16 *>(k_prev);
+    p.palpha = alpha_prev; p.pu = u_prev_or_null;
+    p.pnode_offsets = node_offsets_prev; p.pparent = parent_prev_or_null; p.Tp = total_nodes_prev;
+    p.status = status_word;
+    p.ws = carve_workspace(workspace, dims->batch, total_nodes);
+    p.n_slots = tree_slots_needed(dims->max_nodes);
+    rc = cuda_rc(launch_plan(p, st));
+    if (rc != SPECA_OK) return rc;
+    rc = cuda_rc(launch_pending_check(p, 8, st));
+    if (rc != SPECA_OK) return rc;
+    return cuda_rc(launch_verify_factorized(p, true, st));
 }
 
 }  // extern "C"

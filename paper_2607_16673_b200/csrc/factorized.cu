@@ -30,6 +30,15 @@
 // bandwidth (operand reads by the tensor core, coefficient broadcasts) is the scarce on-chip
 // resource, which is what the two-rows-per-thread epilogue is for.  Every wait is bounded; on
 // expiry the CTA raises SPECA_STATUS_TIMEOUT, drains and exits.
+//
+// Fused commit-and-verify (the delayed state update of Section 5).  A second instantiation
+// adds one role, the warps after the epilogue groups: between the TMA landing a state slice and the tensor core
+// reading it, they advance the slice in place over the pending accepted path,
+//        S <- gamma_A S + sum_{i < A} (gamma_A / gamma_i) u_i k_i^T ,
+// with the u_i the previous verification wrote, and send the slice back to HBM with a TMA
+// store.  The tensor core then reads the committed state, so everything downstream is the
+// plain verification; the state crosses HBM twice per round (one read, one write) instead
+// of three times.
 #include <cuda.h>
 
 #include <type_traits>
@@ -55,6 +64,12 @@ constexpr int kAccCols = 2 * kMaxNodes;        // 128 TMEM columns per tile accu
 constexpr int kPairCols = 2 * kAccCols;        // a unit's two tiles
 constexpr int kTmemCols = 512;                 // two units in flight
 constexpr int kThreads = 14 * 32;
+#ifndef SPECA_UPD_WARPS
+#define SPECA_UPD_WARPS 2
+#endif
+constexpr int kUpdWarps = SPECA_UPD_WARPS;                   // state-update role of the fused kernel
+constexpr int kUpdThreads = kUpdWarps * 32;
+constexpr int kThreadsFused = kThreads + kUpdThreads;
 constexpr int kPrepThreads = 128;
 constexpr int kEpiChunk = 4;                   // nodes per TMEM read in the epilogue
 constexpr int kGramHalf = 32;                  // Gram columns parked per extraction pass
@@ -68,8 +83,13 @@ constexpr int kOffGram = kOffStage + 2 * kStageChunkBytes;
 constexpr int kOffCoef = kOffGram + kGramHalf * kTileRows * 4;
 constexpr int kOffAlpha = kOffCoef + 2 * kMaxNodes * kCoefStride * 4;
 constexpr int kOffBars = kOffAlpha + 2 * kMaxNodes * 4;                   // alpha, beta by position
-constexpr int kOffMisc = kOffBars + 8 * 32;
-constexpr int kSmemBytes = kOffMisc + 64 + 1024;                          // + alignment slack
+constexpr int kOffMisc = kOffBars + 8 * 40;
+constexpr int kOffPendK = kOffMisc + 64;                                  // bf16 keys of the pending path [2][8][d_k + 8]
+constexpr int kOffWalk = kOffPendK + 2 * kMaxDepth * (kDK * 2 + 16);       // per-sequence walk table
+constexpr int kWalkSeqs = 192;                                            // sequences the table holds
+constexpr int kWalkOffs = 0, kWalkPBase = 4 * kWalkSeqs, kWalkPNode = 8 * kWalkSeqs, kWalkN = 16 * kWalkSeqs,
+              kWalkA = 17 * kWalkSeqs;
+constexpr int kSmemBytes = kOffWalk + 18 * kWalkSeqs;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 enum Bar {
@@ -85,9 +105,11 @@ enum Bar {
     kBarAccFull = kBarCoefFree + 2,      // [2] MMA -> epilogue group: the unit's accumulators are complete
     kBarPairFree = kBarAccFull + 2,      // [2] epilogue group -> MMA: accumulator columns released
     kBarDrain = kBarPairFree + 2,        // MMA warp: everything issued has completed
+    kBarUpd,                             // [kStages] fused only: update role -> MMA, slice advanced in place
+    kBarUpdSync = kBarUpd + kStages,     // fused only: rendezvous of the update role's threads
     kBarCount
 };
-static_assert(kBarCount <= 32, "barrier region too small");
+static_assert(kBarCount <= 40, "barrier region too small");
 
 // ----------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
@@ -137,6 +159,9 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
     for (uint32_t it = 0;; ++it) {
         const bool ok = mbar_try_wait(bar, parity);
         if (__any_sync(0xffffffffu, ok)) return true;
+#ifdef SPECA_SPIN_SLEEP
+        __nanosleep(SPECA_SPIN_SLEEP);
+#endif
         if ((it & 255u) == 255u) {
             if (__any_sync(0xffffffffu, *abort_flag != 0)) return false;
             const uint64_t now = global_timer_ns();
@@ -197,6 +222,20 @@ __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int x, i
     asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int y, int z, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// all but the newest N store groups have finished READING shared memory
+template <int N> __device__ __forceinline__ void tma_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// every store group has completed
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -261,6 +300,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
     d |= uint64_t(2) << 61;                              // SWIZZLE_128B
     return d;
 }
+// warp-level D = A B + D, m16n8k8, TF32 operands (bit patterns), fp32 accumulate
+__device__ __forceinline__ void mma_tf32_sync(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 // kind::tf32, fp32 accumulate, both operands K-major, M = 128
 __device__ __forceinline__ uint32_t make_idesc(int n)
 {
@@ -303,27 +350,44 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
 // order, ancestors) is loaded once.  Sequences that failed validation or are empty are
 // skipped.  Every role walks the same list; unit number i of a CTA (unit_seq) uses
 // accumulator pair, coefficient buffer and epilogue group i & 1.
-struct Unit { int grp, hi, u, b, l, h, n, npad, base; };
-struct UnitWalk { int HG, gpl, n_groups, H, B, grid; const int32_t *seq_n; const int32_t *offs; };
+// Fused walk: a is the length of the sequence's pending accepted path; a sequence whose new
+// tree is empty or was rejected still gets its commit (a unit with no nodes).
+struct Unit { int grp, hi, u, b, l, h, n, npad, base, a; };
+// What the walk needs per sequence (node count, offset, pending path) is copied into shared
+// memory when the kernel starts, for the first kWalkSeqs sequences: a global load on the
+// per-unit control path costs a full memory round trip under a saturated HBM.
+struct UnitWalk {
+    int HG, gpl, n_groups, H, B, grid;
+    const int32_t *seq_n; const int32_t *offs; const int32_t *pend;
+    const uint8_t *tab;
+};
 
 __device__ __forceinline__ bool load_group(const UnitWalk &w, int G, Unit &x)
 {
     for (; G < w.n_groups; G += w.grid) {
         const int lb = G / w.gpl;                        // (layer, sequence) pair
         x.b = lb % w.B;
-        x.n = w.seq_n[x.b];
-        if (x.n > 0) {
+        const bool in_tab = x.b < kWalkSeqs;
+        if (in_tab) {
+            x.n = reinterpret_cast<const int8_t *>(w.tab + kWalkN)[x.b];
+            x.a = reinterpret_cast<const int8_t *>(w.tab + kWalkA)[x.b];
+        } else {
+            x.n = w.seq_n[x.b];
+            x.a = w.pend != nullptr ? __ldg(w.pend + x.b * kPendWords) : 0;
+        }
+        if (x.a > 0 && x.n < 0) x.n = 0;
+        if (x.n > 0 || x.a > 0) {
             x.grp = G;
             x.hi = 0;
             x.l = lb / w.B;
             x.h = (G - lb * w.gpl) * w.HG;
             x.u = lb * w.H + x.h;
-            x.npad = (x.n + 15) & ~15;
-            x.base = __ldg(w.offs + x.b);
+            x.npad = x.n > 0 ? (x.n + 15) & ~15 : 16;
+            x.base = in_tab ? reinterpret_cast<const int32_t *>(w.tab + kWalkOffs)[x.b] : __ldg(w.offs + x.b);
             return true;
         }
     }
-    x.n = 0; x.grp = w.n_groups;
+    x.n = 0; x.a = 0; x.grp = w.n_groups;
     return false;
 }
 __device__ __forceinline__ bool first_unit(const UnitWalk &w, Unit &x) { return load_group(w, int(blockIdx.x), x); }
@@ -380,9 +444,9 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
     }
 }
 
-// TP = value tiles per unit (d_v / 128): 1 or 2.
-template <int TP>
-__global__ void __launch_bounds__(kThreads, 1)
+// TP = value tiles per unit (d_v / 128): 1 or 2.  FUSED adds the state-update role.
+template <int TP, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? kThreadsFused : kThreads, 1)
 verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
     // The swizzled operand regions need 1024-byte alignment.  The array is declared with that
@@ -404,7 +468,13 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarFull + s), 1); mbar_init(bar(kBarEmpty + s), 1); }
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar(kBarFull + s), 1);
+            // fused: a slot is free once the tensor core AND the TMA store have read it
+            mbar_init(bar(kBarEmpty + s), FUSED ? 2 : 1);
+            mbar_init(bar(kBarUpd + s), kUpdThreads);
+        }
+        mbar_init(bar(kBarUpdSync), kUpdThreads);
         mbar_init(bar(kBarBReady), kPrepThreads);
         mbar_init(bar(kBarBFree), 1);
         mbar_init(bar(kBarStageReady), 1);
@@ -419,6 +489,19 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         mbar_init(bar(kBarDrain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int b = threadIdx.x; b < p.B && b < kWalkSeqs; b += blockDim.x) {
+        const int n = p.ws.seq_n[b];
+        reinterpret_cast<int8_t *>(smem + kOffWalk + kWalkN)[b] = int8_t(n < 0 ? -1 : n);       // n <= kMaxNodes
+        reinterpret_cast<int32_t *>(smem + kOffWalk + kWalkOffs)[b] = p.node_offsets[b];
+        int a = 0;
+        if (FUSED) {
+            const int32_t *rec = p.ws.pend + b * kPendWords;
+            a = rec[0];
+            reinterpret_cast<int32_t *>(smem + kOffWalk + kWalkPBase)[b] = rec[9];
+            for (int i = 0; i < kMaxDepth; ++i) smem[kOffWalk + kWalkPNode + b * kMaxDepth + i] = uint8_t(rec[1 + i]);
+        }
+        reinterpret_cast<int8_t *>(smem + kOffWalk + kWalkA)[b] = int8_t(a);
+    }
     if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
     tc_fence_before();
     __syncthreads();
@@ -430,6 +513,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     walk.n_groups = int(fp.n_units / fp.heads_per_group);
     walk.H = p.H; walk.B = p.B; walk.grid = int(gridDim.x);
     walk.seq_n = p.ws.seq_n; walk.offs = p.node_offsets;
+    walk.pend = FUSED ? p.ws.pend : nullptr;
+    walk.tab = smem + kOffWalk;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
@@ -440,7 +525,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
             // the value rows of this unit's nodes are read by the epilogue with plain loads a
             // couple of units from now: pull them into L2 meanwhile
-            if (lane == 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
+            if (lane == 0 && x.n > 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
             for (int t = 0; t < TP && ok; ++t) {
                 // tile t of a unit holds its value rows t, t + TP, t + 2 TP, ... (interleaved tiles:
                 // an epilogue thread then owns TP ADJACENT value rows, one per tile)
@@ -466,6 +551,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
         uint32_t it = 0, unit_seq = 0;
+        int pending_slot = -1;                                   // fused: slot whose store may still be reading it
         Unit x;
         bool ok = true;
         const uint32_t bop = sbase + kOffBop, stage = sbase + kOffStage;
@@ -505,7 +591,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 for (int c = 0; c < kChunks; ++c, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
-                    if (!(ok = WAIT(4, bar(kBarFull + s), ph))) break;
+                    if (!(ok = WAIT(4, bar((FUSED ? kBarUpd : kBarFull) + s), ph))) break;
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t sa = sbase + kOffRing + s * kStageBytes;
@@ -514,6 +600,23 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                             mma_tf32(acc + t * kAccCols, make_desc(sa + k * 32),
                                      make_desc(bop + c * kBopChunkBytes + k * 32), idm, (c | k) != 0);
                         mma_commit(bar(kBarEmpty + s));
+                        if (FUSED) {
+                            // send the advanced slice back to HBM; a slot is released one store later,
+                            // when its own store has certainly finished reading it
+                            if (x.a > 0) {
+                                tma_store_3d(&s0_map, c * kChunkK, t, x.u * kTileRows, sa);
+                                tma_store_wait_read<1>();
+                                if (pending_slot >= 0) mbar_arrive(bar(kBarEmpty + pending_slot));
+                                pending_slot = s;
+                            } else {
+                                if (pending_slot >= 0) {
+                                    tma_store_wait_read<0>();
+                                    mbar_arrive(bar(kBarEmpty + pending_slot));
+                                    pending_slot = -1;
+                                }
+                                mbar_arrive(bar(kBarEmpty + s));
+                            }
+                        }
                     }
                     __syncwarp();
                 }
@@ -526,6 +629,13 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (have) ok = issue_gram(unit_seq, x.npad);
         }
         PROF_STORE()
+        if (FUSED && lane == 0) {
+            if (pending_slot >= 0) {
+                tma_store_wait_read<0>();
+                mbar_arrive(bar(kBarEmpty + pending_slot));
+            }
+            tma_store_wait_all();
+        }
         // everything this warp issued must have completed before TMEM is released
         if (lane == 0) mma_commit(bar(kBarDrain));
         __syncwarp();
@@ -734,7 +844,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             cur_lo = node_lo; cur_hi = node_hi;
         }
         PROF_STORE()
-    } else {
+    } else if (warp < 14) {
         // ------------------------------------------------------------- epilogue groups
         const int grp = (warp - 6) >> 2;
         const int row = 32 * (warp & 3) + lane;
@@ -758,6 +868,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         const VPack *vraw = reinterpret_cast<const VPack *>(p.v);
         // value rows of the first chunk of a unit, fetched ahead (node order from the plan)
         auto fetch_first_values = [&](const Unit &y) {
+            if (y.n == 0) return;                            // commit-only unit: no records to read
             const int rec0 = (y.l * p.T + y.base) * p.H + y.h;
 #pragma unroll
             for (int i = 0; i < kEpiChunk; ++i) {
@@ -829,7 +940,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             };
             // Software pipeline, one chunk deep: buffer A is processed while buffer B (the next
             // chunk's TMEM columns and value rows) is in flight; B is then moved into A.
-            load_tmem(0, RA, GA);
+            if (n > 0) load_tmem(0, RA, GA);
 #pragma unroll 1
             for (int p0 = 0; p0 < n; p0 += kEpiChunk) {
                 tmem_ld_wait();
@@ -855,6 +966,199 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (have) fetch_first_values(x);
         }
         PROF_STORE()
+    } else if (FUSED) {
+        // ------------------------------------------------------------- state update (fused commit)
+        // The pending update of a slice, S <- gA S + W Kp (W[r][i] = (gamma_A / gamma_i) u_i[r],
+        // Kp[i][c] = k_i[c], i < A <= 8), is a rank-8 product: each warp applies it to its rows
+        // with warp-level m16n8k8 TF32 MMAs whose accumulator fragment is the slice itself, read
+        // from and written back to the shared-memory slot.  Keys are bf16 (exact in TF32); W is
+        // split into a TF32 head and tail (two MMAs), so the products carry fp32 accuracy and the
+        // accumulation is fp32.  The cost does not depend on A and the only shared-memory round
+        // trip per batch of rows is the slice itself.
+        // Lane l keeps the index and the gate of path node l & 7; the others get them by shuffle.
+        // Everything global is fetched one unit (keys, gates) or one tile (u) ahead, and the node
+        // indices are re-read only when the sequence changes: a load whose address depends on
+        // another load costs this role a full memory round trip under a saturated HBM.
+        const int ut = threadIdx.x - kThreads;
+        const int uw = ut >> 5;                                  // warp of the role
+        const int g = lane >> 2, t4 = lane & 3;                  // MMA fragment coordinates
+        const int li = lane & 7;
+        constexpr int kRowsPerWarp = kTileRows / kUpdWarps, kMT = kRowsPerWarp / 16;
+        const int rowbase = uw * kRowsPerWarp;
+        constexpr int kKeyStride = kDK * 2 + 16;                 // bytes per staged key (bank-conflict padding)
+        constexpr int kKeyBuf = kMaxDepth * kKeyStride;
+        constexpr int kKeyPieces = kMaxDepth * 16 / kUpdThreads; // 16-byte pieces each thread copies per unit
+        int node_c = 0, node_n = 0, grp_n = -1;
+        float alpha_c = 1.f, alpha_n = 1.f;
+        float wn[kMT][4];
+#pragma unroll
+        for (int m = 0; m < kMT; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) wn[m][e] = 0.f;
+        auto fetch_unit = [&](const Unit &y, int buf) {
+            if (y.a == 0) return;
+            if (y.b < kWalkSeqs) {
+                node_n = reinterpret_cast<const int32_t *>(smem + kOffWalk + kWalkPBase)[y.b] +
+                         int(smem[kOffWalk + kWalkPNode + y.b * kMaxDepth + li]);
+            } else if (y.grp != grp_n) {
+                grp_n = y.grp;
+                node_n = __ldg(p.ws.pend + y.b * kPendWords + 9) + (li < y.a ? __ldg(p.ws.pend + y.b * kPendWords + 1 + li) : 0);
+            }
+            alpha_n = li < y.a ? __ldg(p.palpha + (size_t(y.l) * p.Tp + node_n) * p.H + y.h) : 1.f;
+#pragma unroll
+            for (int q = 0; q < kKeyPieces; ++q) {
+                const int piece = ut * kKeyPieces + q;           // 0..127: node piece >> 4, 16-byte piece & 15
+                const int kn = __shfl_sync(0xffffffffu, node_n, piece >> 4);
+                if ((piece >> 4) < y.a) {
+                    const __nv_bfloat16 *src = p.pk + ((size_t(y.l) * p.Tp + kn) * p.H + y.h) * kDK + (piece & 15) * 8;
+                    cp_async_16(sbase + kOffPendK + buf * kKeyBuf + (piece >> 4) * kKeyStride + (piece & 15) * 16, src);
+                }
+            }
+        };
+        // u of the pending nodes in A-fragment order: [m][0..3] = (row g, node t4), (row g + 8, node t4),
+        // (row g, node t4 + 4), (row g + 8, node t4 + 4) of m-tile m; zero past the end of the path
+        auto fetch_tile = [&](const Unit &y, int t, int node_reg) {
+            if (y.a == 0) return;
+            const int n0 = __shfl_sync(0xffffffffu, node_reg, t4), n1 = __shfl_sync(0xffffffffu, node_reg, t4 + 4);
+            const float *u0 = p.pu + ((size_t(y.l) * p.Tp + n0) * p.H + y.h) * p.DV + t;
+            const float *u1 = p.pu + ((size_t(y.l) * p.Tp + n1) * p.H + y.h) * p.DV + t;
+#pragma unroll
+            for (int m = 0; m < kMT; ++m) {
+                const int r0 = (rowbase + 16 * m + g) * TP, r1 = r0 + 8 * TP;
+                wn[m][0] = t4 < y.a ? __ldg(u0 + r0) : 0.f;
+                wn[m][1] = t4 < y.a ? __ldg(u0 + r1) : 0.f;
+                wn[m][2] = t4 + 4 < y.a ? __ldg(u1 + r0) : 0.f;
+                wn[m][3] = t4 + 4 < y.a ? __ldg(u1 + r1) : 0.f;
+            }
+        };
+
+        uint32_t it = 0, sync_no = 0, useq = 0;
+        Unit x, nx;
+        bool ok = true;
+        bool have = first_unit(walk, x);
+        if (have) {
+            fetch_unit(x, 0);
+            node_c = node_n; alpha_c = alpha_n;
+            fetch_tile(x, 0, node_c);
+        }
+        PROF_DECL
+        auto group_sync = [&]() -> bool {
+            mbar_arrive(bar(kBarUpdSync));
+            const bool r = wait_fast(bar(kBarUpdSync), sync_no & 1, abort_flag);
+            ++sync_no;
+            return r;
+        };
+        for (; have && ok; ++useq) {
+            const int A = x.a;
+            const int buf = useq & 1;
+            PROF_MARK()
+            // this thread's key pieces of unit x have landed; after the rendezvous everybody's are
+            // visible and everybody has left the previous unit (whose key buffer is refilled below)
+            cp_async_wait_all();
+            if (!(ok = group_sync())) break;
+            // my_ratio = product of alpha over the path nodes after node li; gA over all of them
+            float my_ratio = 1.f, gA = 1.f;
+#pragma unroll
+            for (int j = 0; j < kMaxDepth; ++j) {
+                const float aj = __shfl_sync(0xffffffffu, alpha_c, j);
+                if (j < A) {
+                    gA *= aj;
+                    if (j > li) my_ratio *= aj;
+                }
+            }
+            const float ratio0 = __shfl_sync(0xffffffffu, my_ratio, t4), ratio1 = __shfl_sync(0xffffffffu, my_ratio, t4 + 4);
+            PROF_SEG(1)
+            nx = x;
+            const bool have_next = next_unit(walk, nx);
+            if (have_next) fetch_unit(nx, buf ^ 1);
+            PROF_SEG(2)
+            for (int t = 0; t < TP && ok; ++t) {
+                // A fragments of this tile: W = ratio * u
+                float w[kMT][4];
+#pragma unroll
+                for (int m = 0; m < kMT; ++m) {
+                    w[m][0] = ratio0 * wn[m][0]; w[m][1] = ratio0 * wn[m][1];
+                    w[m][2] = ratio1 * wn[m][2]; w[m][3] = ratio1 * wn[m][3];
+                }
+                PROF_SEG(3)
+                if (t + 1 < TP) fetch_tile(x, t + 1, node_c);
+                else if (have_next) fetch_tile(nx, 0, node_n);
+                PROF_SEG(4)
+                for (int c = 0; c < kChunks; ++c, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1;
+                    if (!(ok = WAIT(0, bar(kBarFull + s), ph))) break;
+                    PROF_MARK()
+                    if (A > 0) {
+                        uint8_t *slot = smem + kOffRing + s * kStageBytes;
+                        // B fragments: keys t4 and t4 + 4 at column 8 n + g of this chunk
+                        const uint8_t *kb = smem + kOffPendK + buf * kKeyBuf + (c * kChunkK + g) * 2;
+                        uint32_t b0[4], b1[4];
+#pragma unroll
+                        for (int n = 0; n < 4; ++n) {
+                            const uint32_t lo = *reinterpret_cast<const unsigned short *>(kb + t4 * kKeyStride + n * 16);
+                            const uint32_t hi = *reinterpret_cast<const unsigned short *>(kb + (t4 + 4) * kKeyStride + n * 16);
+                            b0[n] = t4 < A ? lo << 16 : 0u;
+                            b1[n] = t4 + 4 < A ? hi << 16 : 0u;
+                        }
+#pragma unroll
+                        for (int mb = 0; mb < kMT; mb += 2) {
+                            // accumulator fragments of two m-tiles: rows R, R + 8; columns 8 n + 2 t4, + 1
+                            float cf[2][4][4];
+#pragma unroll
+                            for (int m2 = 0; m2 < 2; ++m2) {
+                                const int R = rowbase + 16 * (mb + m2) + g;
+#pragma unroll
+                                for (int n = 0; n < 4; ++n) {
+                                    const uint32_t off = ((uint32_t(2 * n + (t4 >> 1)) ^ uint32_t(R & 7)) << 4) | uint32_t((t4 & 1) * 8);
+                                    const float2 v0 = *reinterpret_cast<const float2 *>(slot + R * 128 + off);
+                                    const float2 v1 = *reinterpret_cast<const float2 *>(slot + (R + 8) * 128 + off);
+                                    cf[m2][n][0] = v0.x; cf[m2][n][1] = v0.y; cf[m2][n][2] = v1.x; cf[m2][n][3] = v1.y;
+                                }
+                            }
+#pragma unroll
+                            for (int m2 = 0; m2 < 2; ++m2) {
+                                uint32_t ah[4], al[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float wv = w[mb + m2][e];
+                                    ah[e] = __float_as_uint(wv) & 0xffffe000u;
+                                    al[e] = __float_as_uint(wv - __uint_as_float(ah[e]));
+                                }
+#pragma unroll
+                                for (int n = 0; n < 4; ++n) {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) cf[m2][n][e] *= gA;
+                                    mma_tf32_sync(cf[m2][n], ah, b0[n], b1[n]);
+                                    mma_tf32_sync(cf[m2][n], al, b0[n], b1[n]);
+                                }
+                            }
+#pragma unroll
+                            for (int m2 = 0; m2 < 2; ++m2) {
+                                const int R = rowbase + 16 * (mb + m2) + g;
+#pragma unroll
+                                for (int n = 0; n < 4; ++n) {
+                                    const uint32_t off = ((uint32_t(2 * n + (t4 >> 1)) ^ uint32_t(R & 7)) << 4) | uint32_t((t4 & 1) * 8);
+                                    *reinterpret_cast<float2 *>(slot + R * 128 + off) = make_float2(cf[m2][n][0], cf[m2][n][1]);
+                                    *reinterpret_cast<float2 *>(slot + (R + 8) * 128 + off) = make_float2(cf[m2][n][2], cf[m2][n][3]);
+                                }
+                            }
+                        }
+                        PROF_SEG(5)
+                        fence_proxy_async();                 // the tensor core and the TMA store read this slice
+                    }
+                    mbar_arrive(bar(kBarUpd + s));
+                    PROF_SEG(7)
+                    PROF_SEG(6)
+                }
+            }
+            x = nx;
+            have = have_next;
+            node_c = node_n;
+            alpha_c = alpha_n;
+        }
+        PROF_STORE()
+        cp_async_wait_all();
     }
 
     tc_fence_before();
@@ -891,7 +1195,7 @@ bool factorized_supported(const speca_dims *d)
            d->max_depth <= kMaxDepth;
 }
 
-int launch_verify_factorized(const Params &p, cudaStream_t st)
+int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st)
 {
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return int(cudaErrorNotSupported);
@@ -940,10 +1244,16 @@ int launch_verify_factorized(const Params &p, cudaStream_t st)
     }
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(verify_factorized_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(verify_factorized_kernel<1, false>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(verify_factorized_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(verify_factorized_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(verify_factorized_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(verify_factorized_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kSmemBytes);
         if (e != cudaSuccess) return int(e);
         attr_set = true;
@@ -954,8 +1264,13 @@ int launch_verify_factorized(const Params &p, cudaStream_t st)
     fp.heads_per_group = (p.H % 4 == 0) ? 4 : (p.H % 2 == 0 ? 2 : 1);
     const long n_groups = n_units / fp.heads_per_group;
     const int grid = int(n_groups < sm_count ? n_groups : sm_count);
-    if (p.DV == kTileRows) verify_factorized_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-    else verify_factorized_kernel<2><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+    if (fused) {
+        if (p.DV == kTileRows) verify_factorized_kernel<1, true><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, true><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+    } else {
+        if (p.DV == kTileRows) verify_factorized_kernel<1, false><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, false><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+    }
     return int(cudaGetLastError());
 }
 

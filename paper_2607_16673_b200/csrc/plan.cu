@@ -192,7 +192,49 @@ accept_kernel(int32_t B, int32_t max_depth, const int32_t *__restrict__ node_off
     }
 }
 
+// Pending accepted paths of the fused commit-and-verify call, one thread per sequence:
+// the same checks the stand-alone commit makes (length, node range, parent chain when the
+// parent array is given), plus a node count within max_nodes.  A bad path is reported and
+// recorded with length 0, so the sequence's state is not advanced; a good one is stored as
+// local node indices (words 1..8) and the sequence's offset in the previous draft's packed
+// arrays (word 9).
+__global__ void __launch_bounds__(128)
+pending_check_kernel(int32_t B, int32_t Tp, int32_t max_depth, int32_t max_len, int32_t max_nodes,
+                     const int32_t *__restrict__ pnode_offsets, const int32_t *__restrict__ pparent,
+                     const int32_t *__restrict__ path_idx, const int32_t *__restrict__ path_len,
+                     int32_t *__restrict__ pend, int32_t *status)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int32_t *rec = pend + b * kPendWords;
+    const int len = path_len[b];
+    const int base = pnode_offsets[b];
+    const int n = pnode_offsets[b + 1] - base;
+    int fault = 0;
+    if (len < 0 || len > max_depth || len > max_len) fault = SPECA_STATUS_TOO_DEEP;
+    else if (len > 0 && (base < 0 || n < 0 || base + n > Tp)) fault = SPECA_STATUS_BAD_OFFSETS;
+    else if (len > 0 && n > max_nodes) fault = SPECA_STATUS_TOO_MANY;
+    int prev = -1;
+    for (int d = 0; d < len && !fault; ++d) {
+        const int t = path_idx[b * max_depth + d];
+        if (t < 0 || t >= n) fault = SPECA_STATUS_BAD_PATH;
+        else if (pparent != nullptr && pparent[base + t] != prev) fault = SPECA_STATUS_BAD_PATH;
+        if (!fault) rec[1 + d] = t;
+        prev = t;
+    }
+    if (fault) atomicOr(status, fault);
+    rec[0] = fault ? 0 : len;
+    rec[9] = base;
+}
+
 }  // namespace
+
+int launch_pending_check(const Params &p, int max_len, cudaStream_t st)
+{
+    pending_check_kernel<<<(p.B + 127) / 128, 128, 0, st>>>(p.B, p.Tp, p.max_depth, max_len, p.max_nodes, p.pnode_offsets,
+                                                            p.pparent, p.path_idx, p.path_len, p.ws.pend, p.status);
+    return int(cudaGetLastError());
+}
 
 int launch_plan(const Params &p, cudaStream_t st)
 {

@@ -16,10 +16,14 @@ namespace speca {
 //   [2048, 2048 + 4*Bpad)        seq_n[b]: node count of sequence b, or -1 if the
 //                                sequence failed validation and must be skipped
 //   then int32 arrays of Tpad words: plan[T], depth[T], anc[T][4]
+//   after the kNodeWords node arrays, used only by the fused commit-and-verify call:
+//   pend[B][kPendWords]: validated length of the pending accepted path, its local node
+//   indices, and the sequence's offset in the previous draft's packed arrays
 // Every region starts on a 256-byte boundary.
 // ---------------------------------------------------------------------------
 constexpr size_t kCtrlBytes = 2048;
 constexpr int kNodeWords = 16;          // int32 words of scratch reserved per packed node
+constexpr int kPendWords = 12;          // per sequence: path length, 8 local node indices, offset, spare
 
 __host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -29,11 +33,13 @@ struct Workspace {
     int32_t *plan;      // [T]   packed schedule entries, in processing order per sequence
     int32_t *depth;     // [T]   depth computed from parent[]
     int32_t *anc;       // [T][4] per node: depth | position << 8, ancestor node indices by level (8 bytes), spare
+    int32_t *pend;      // [B][kPendWords] pending accepted path (fused commit-and-verify only)
 };
 
 inline size_t workspace_bytes(int32_t batch, int32_t total_nodes)
 {
-    return kCtrlBytes + align256(size_t(batch) * 4) + align256(size_t(total_nodes) * 4) * kNodeWords;
+    return kCtrlBytes + align256(size_t(batch) * 4) + align256(size_t(total_nodes) * 4) * kNodeWords +
+           align256(size_t(batch) * kPendWords * 4);
 }
 
 inline Workspace carve_workspace(void *base, int32_t batch, int32_t total_nodes)
@@ -48,6 +54,7 @@ inline Workspace carve_workspace(void *base, int32_t batch, int32_t total_nodes)
     w.plan = reinterpret_cast<int32_t *>(p);
     w.depth = reinterpret_cast<int32_t *>(p + tb);
     w.anc = reinterpret_cast<int32_t *>(p + 2 * tb);
+    w.pend = reinterpret_cast<int32_t *>(p + kNodeWords * tb);
     return w;
 }
 
@@ -73,6 +80,11 @@ struct Params {
     float *o, *u;
     const int32_t *node_offsets, *parent, *depth_in;
     const int32_t *path_idx, *path_len;
+    // pending commit of the fused call: records of the previous draft (keys, gates, u) and its packing
+    const __nv_bfloat16 *pk;
+    const float *palpha, *pu;
+    const int32_t *pnode_offsets, *pparent;
+    int32_t Tp;
     int32_t *status;
     Workspace ws;
     int32_t n_slots;             // on-chip state slots available to the tree walk
@@ -84,7 +96,8 @@ int launch_decode(const Params &p, int d_k, cudaStream_t st);
 int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
 int launch_commit(const Params &p, int d_k, cudaStream_t st);
 bool factorized_supported(const speca_dims *d);
-int launch_verify_factorized(const Params &p, cudaStream_t st);
+int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st);
+int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
 int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
                   const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
                   int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,
