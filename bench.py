@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-fused", action="store_true", help="skip the fused commit-and-verify leg")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling only)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling only)")
     return ap.parse_args()
@@ -313,6 +314,11 @@ def run_speca(args):
     dec_bytes = L * B * H * (2 * 4 * dk * dv + 4 * dk + 2 * dv + 8 + 4 * dv)
     del S_dec
 
+    # --- the same rounds with the commit delayed into the next round's verification ----
+    fused = None
+    if not args.no_fused:
+        fused = run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, dist if world > 1 else None, dev)
+
     # --- end to end with host buffers (C ABI fed from pinned host memory) ---------
     e2e = None
     if not args.no_e2e and rank == 0:
@@ -352,6 +358,7 @@ def run_speca(args):
                         "token_layers_per_s": B * L / (dec_ms * 1e-3),
                         "note": "one autoregressive token per sequence at the same batch"},
         "gpu_launches": 4 * K,
+        "fused": fused,
         "clocks": clocks,
         "e2e": e2e,
     }
@@ -360,6 +367,68 @@ def run_speca(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, dist, dev):
+    """The same rounds through speca_commit_verify_tree: round r verifies its draft from the state
+    with round r-1's accepted paths applied on chip (the state is read once and written once per
+    round), then runs greedy acceptance.  Reported beside the headline, not instead of it."""
+    import torch
+    L, B, H, dk, dv = dims.n_layers, dims.batch, dims.heads, dims.d_k, dims.d_v
+    Tmax = max(p["T"] for p in pool)
+    u_buf = [torch.empty(L * Tmax * H * dv, dtype=torch.float32, device=dev) for _ in range(2)]
+    paths = [(torch.zeros(B, 8, dtype=torch.int32, device=dev), torch.zeros(B, dtype=torch.int32, device=dev))
+             for _ in range(2)]
+    next_tok = torch.zeros(B, dtype=torch.int32, device=dev)
+    view = lambda buf, T: buf[: L * T * H * dv].view(L, T, H, dv)
+
+    def step(i):
+        p = pool[i % POOL]
+        T = p["T"]
+        pi, pl = paths[i & 1]
+        prev, (ppi, ppl) = None, paths[(i - 1) & 1]
+        if i > 0:
+            pp = pool[(i - 1) % POOL]
+            prev = dict(k=pp["k"], v=pp["v"], alpha=pp["alpha"], beta=pp["beta"], u=view(u_buf[(i - 1) & 1], pp["T"]),
+                        node_offsets=pp["d_offs"], total_nodes=pp["T"], parent=pp["d_parent"])
+        speca.commit_verify_tree(dims, S, prev, ppi, ppl, p["q"], p["k"], p["v"], p["alpha"], p["beta"], p["d_offs"], T,
+                                 p["d_parent"], p["d_depth"], view(o_buf, T), view(u_buf[i & 1], T), ws, status)
+        speca.greedy_accept(B, 8, p["d_offs"], p["d_parent"], p["d_draft"], p["d_target"], p["d_root"], pi, pl,
+                            next_tok, status)
+
+    W, K = max(3, args.warmup), args.steps
+    for i in range(W):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(W, W + K):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    assert int(status.item()) == 0, f"device status word {int(status.item())}"
+    tokens = sum(pool[i % POOL]["T"] for i in range(W, W + K))
+    # algorithmic bytes: state read once, written once where something is committed, records in, o out,
+    # records of the accepted nodes; the u rows written and re-read are not counted
+    Sb = 4 * dk * dv
+    nbytes = 0
+    for i in range(W, W + K):
+        p, pp = pool[i % POOL], pool[(i - 1) % POOL]
+        nbytes += L * B * H * Sb + int(np.count_nonzero(pp["path_len"])) * L * H * Sb
+        nbytes += p["T"] * L * H * (4 * dk + 2 * dv + 8 + 4 * dv) + int(pp["path_len"].sum()) * L * H * (2 * dk + 2 * dv + 8)
+    if dist is not None:
+        tt = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        cnt = torch.tensor([tokens, nbytes], device=dev, dtype=torch.float64)
+        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
+        ms, tokens, nbytes = float(tt[0]), float(cnt[0]), float(cnt[1])
+    peak, peak_kind = measured_peak_gbs()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"value": tokens * L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / K, "steps": K, "gpu_launches": 4 * K,
+            "algorithmic_gbs": gbs, "frac_of_peak": gbs / peak, "peak_kind": f"of {peak_kind}",
+            "note": "speca_commit_verify_tree + speca_greedy_accept per round; the commit of round r runs inside the "
+                    "verification of round r+1 (state read once and written once per round)"}
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant

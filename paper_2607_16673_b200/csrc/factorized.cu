@@ -55,6 +55,14 @@ constexpr int kChunkK = 32;                    // floats per 128-byte swizzle ro
 constexpr int kChunks = kDK / kChunkK;         // 4 K-chunks per tile
 constexpr int kStageBytes = kTileRows * 128;   // 16 KiB per (tile, K-chunk)
 constexpr int kStages = 6;
+#ifndef SPECA_POLL_NS
+#define SPECA_POLL_NS 100
+#endif
+#ifndef SPECA_FUSED_STAGES
+#define SPECA_FUSED_STAGES 5
+#endif
+constexpr int kStagesFused = SPECA_FUSED_STAGES;                // the fused kernel reads the state at half its total traffic: a
+                                               // shallower ring suffices, the other two slots hold the pending u rows
 constexpr int kMaxNodes = 64;                  // nodes per sequence handled by this route
 constexpr int kMaxDepth = 8;
 constexpr int kBopRows = 2 * kMaxNodes;        // [K;Q] rows
@@ -85,7 +93,14 @@ constexpr int kOffAlpha = kOffCoef + 2 * kMaxNodes * kCoefStride * 4;
 constexpr int kOffBars = kOffAlpha + 2 * kMaxNodes * 4;                   // alpha, beta by position
 constexpr int kOffMisc = kOffBars + 8 * 40;
 constexpr int kOffPendK = kOffMisc + 64;                                  // bf16 keys of the pending path [2][8][d_k + 8]
-constexpr int kOffWalk = kOffPendK + 2 * kMaxDepth * (kDK * 2 + 16);       // per-sequence walk table
+constexpr int kKeyStride = kDK * 2 + 16;                                   // bytes per staged pending key (bank padding)
+constexpr int kKeyBuf = kMaxDepth * kKeyStride;
+constexpr int kOffWalk = kOffPendK + 2 * kKeyBuf;                          // per-sequence walk table
+// fused kernel: u rows of the pending path, [2][8][256 + 16] fp32, in ring slots 4 and 5
+constexpr int kOffPendU = kOffRing + kStagesFused * kStageBytes;
+constexpr int kPendUStride = (2 * kTileRows + (kStagesFused <= 4 ? 16 : 0)) * 4;
+constexpr int kPendUBuf = kMaxDepth * kPendUStride;
+static_assert(2 * kPendUBuf <= (kStages - kStagesFused) * kStageBytes, "pending u rows do not fit the spare ring slots");
 constexpr int kWalkSeqs = 192;                                            // sequences the table holds
 constexpr int kWalkOffs = 0, kWalkPBase = 4 * kWalkSeqs, kWalkPNode = 8 * kWalkSeqs, kWalkN = 16 * kWalkSeqs,
               kWalkA = 17 * kWalkSeqs;
@@ -106,7 +121,8 @@ enum Bar {
     kBarPairFree = kBarAccFull + 2,      // [2] epilogue group -> MMA: accumulator columns released
     kBarDrain = kBarPairFree + 2,        // MMA warp: everything issued has completed
     kBarUpd,                             // [kStages] fused only: update role -> MMA, slice advanced in place
-    kBarUpdSync = kBarUpd + kStages,     // fused only: rendezvous of the update role's threads
+    kBarPendFull = kBarUpd + kStages,    // [2] fused only: TMA producer -> update role, pending u rows and keys staged
+    kBarPendFree = kBarPendFull + 2,     // [2] fused only: update role -> TMA producer
     kBarCount
 };
 static_assert(kBarCount <= 40, "barrier region too small");
@@ -137,6 +153,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// non-blocking probe of a barrier phase
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -222,12 +251,18 @@ __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int x, i
     asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int y, int z, uint32_t src)
+// untiled bulk copy global -> shared (both addresses and the size multiples of 16 bytes)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_3d_nocommit(const CUtensorMap *map, int x, int y, int z, uint32_t src)
 {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
                  ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src)
                  : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 // all but the newest N store groups have finished READING shared memory
 template <int N> __device__ __forceinline__ void tma_store_wait_read()
@@ -470,11 +505,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         *abort_flag = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarFull + s), 1);
-            // fused: a slot is free once the tensor core AND the TMA store have read it
-            mbar_init(bar(kBarEmpty + s), FUSED ? 2 : 1);
+            mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarUpd + s), kUpdThreads);
         }
-        mbar_init(bar(kBarUpdSync), kUpdThreads);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarPendFull + i), 1); mbar_init(bar(kBarPendFree + i), kUpdThreads); }
         mbar_init(bar(kBarBReady), kPrepThreads);
         mbar_init(bar(kBarBFree), 1);
         mbar_init(bar(kBarStageReady), 1);
@@ -508,6 +542,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    constexpr int NS = FUSED ? kStagesFused : kStages;            // ring depth in use
     UnitWalk walk;
     walk.HG = fp.heads_per_group; walk.gpl = p.H / fp.heads_per_group;
     walk.n_groups = int(fp.n_units / fp.heads_per_group);
@@ -516,7 +551,126 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     walk.pend = FUSED ? p.ws.pend : nullptr;
     walk.tab = smem + kOffWalk;
 
-    if (warp == 0) {
+    if (warp == 0 && FUSED) {
+        // ------------------------------------------------------------- TMA producer of the fused kernel
+        // Besides loading state slices it sends the advanced slices back: a TMA store needs a good
+        // fraction of a microsecond to read its 16 KiB out of shared memory under load, so nobody
+        // may block on one.  The warp keeps two cursors over the same sequence of slices, one for
+        // loads and one (behind it) for stores, and serves whichever is ready; a slot is reloaded
+        // once the tensor core has read it and the store of its previous content has read it.
+        // Stores are committed one bulk group per slice (an empty group for slices of units with
+        // nothing pending), so group age equals slice age.
+        uint32_t it = 0, ist = 0, pseq = 0;                      // slices loaded, slices stored, staged units
+        Unit x, nx, xs;                                          // unit being loaded, the one after it, unit being stored
+        int js = 0;                                              // slice of xs the store cursor is at
+        bool ok = true;
+        auto stage_pending = [&](const Unit &y) -> bool {
+            if (y.a == 0) return true;
+            const int pb = pseq & 1;
+            if (!wait_fast(bar(kBarPendFree + pb), ((pseq >> 1) & 1) ^ 1, abort_flag)) return false;
+            if (lane == 0) mbar_arrive_expect_tx(bar(kBarPendFull + pb), uint32_t(y.a) * uint32_t(p.DV * 4 + kDK * 2));
+            __syncwarp();
+            if (lane < y.a) {
+                const int node = y.b < kWalkSeqs
+                    ? reinterpret_cast<const int32_t *>(smem + kOffWalk + kWalkPBase)[y.b] +
+                          int(smem[kOffWalk + kWalkPNode + y.b * kMaxDepth + lane])
+                    : __ldg(p.ws.pend + y.b * kPendWords + 9) + __ldg(p.ws.pend + y.b * kPendWords + 1 + lane);
+                const size_t rec = (size_t(y.l) * p.Tp + node) * p.H + y.h;
+                bulk_load(sbase + kOffPendU + pb * kPendUBuf + lane * kPendUStride, p.pu + rec * p.DV, uint32_t(p.DV * 4),
+                          bar(kBarPendFull + pb));
+                bulk_load(sbase + kOffPendK + pb * kKeyBuf + lane * kKeyStride, p.pk + rec * kDK, uint32_t(kDK * 2),
+                          bar(kBarPendFull + pb));
+            }
+            ++pseq;
+            return true;
+        };
+        // store (or skip) slice ist, which the update role has finished, and advance the store cursor
+        auto issue_store = [&]() {
+            if (lane == 0) {
+                if (xs.a > 0)
+                    tma_store_3d_nocommit(&s0_map, (js % kChunks) * kChunkK, js / kChunks, xs.u * kTileRows,
+                                          sbase + kOffRing + (ist % NS) * kStageBytes);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            __syncwarp();
+            ++ist;
+            if (++js == TP * kChunks) { js = 0; next_unit(walk, xs); }
+        };
+        auto updated = [&](uint32_t i, bool blocking) -> int {   // 1 ready, 0 not yet, -1 abort
+            if (xs.a == 0) return 1;
+            const uint32_t b = bar(kBarUpd + i % NS), ph = (i / NS) & 1;
+            if (!blocking) return __all_sync(0xffffffffu, mbar_test_wait(b, ph)) ? 1 : 0;
+            return wait_fast(b, ph, abort_flag) ? 1 : -1;
+        };
+        bool have = first_unit(walk, x);
+        xs = x;
+        if (have) ok = stage_pending(x);
+        for (; have && ok; x = nx) {
+            nx = x;
+            const bool have_next = next_unit(walk, nx);
+            have = have_next;
+            if (lane == 0 && x.n > 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
+            for (int j = 0; j < TP * kChunks && ok; ++j, ++it) {
+                // halfway through the unit the update role has left the unit before it, whose
+                // staging buffer the next unit's pending path takes
+                if (have_next && j == TP * kChunks / 2 && !(ok = stage_pending(nx))) break;
+                const int s = it % NS;
+                if (it >= uint32_t(NS)) {
+                    // the slot's previous content (slice it - NS) must have been stored ...
+                    while (ok && ist <= it - NS) {
+                        if (updated(ist, true) < 0) ok = false;
+                        else issue_store();
+                    }
+                    if (!ok) break;
+                    // ... and that store must have read it: at most ist - 1 - (it - NS) younger groups pending
+                    if (lane == 0) {
+                        switch (int(ist - 1 - (it - NS))) {
+                        case 0: tma_store_wait_read<0>(); break;
+                        case 1: tma_store_wait_read<1>(); break;
+                        case 2: tma_store_wait_read<2>(); break;
+                        case 3: tma_store_wait_read<3>(); break;
+                        default: tma_store_wait_read<4>(); break;
+                        }
+                    }
+                    __syncwarp();
+                }
+                // wait for the tensor core to release the slot, serving stores that become ready meanwhile
+                {
+                    const uint32_t be = bar(kBarEmpty + s), pe = ((it / NS) & 1) ^ 1;
+                    uint64_t t0 = 0;
+                    for (uint32_t spin = 0; ok; ++spin) {
+                        if (__all_sync(0xffffffffu, mbar_test_wait(be, pe))) break;
+                        if (ist < it && updated(ist, false) == 1) issue_store();
+                        else __nanosleep(SPECA_POLL_NS);         // nothing to do: leave the issue slots to the other warps
+                        if ((spin & 255u) == 255u) {
+                            if (__any_sync(0xffffffffu, *abort_flag != 0)) ok = false;
+                            const uint64_t now = global_timer_ns();
+                            if (t0 == 0) t0 = now;
+                            if (__any_sync(0xffffffffu, now - t0 > kWaitLimitNs)) { *abort_flag = 1; ok = false; }
+                        }
+                    }
+                    if (!ok) break;
+                }
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
+                    tma_load_3d(sbase + kOffRing + s * kStageBytes, &s0_map, (j % kChunks) * kChunkK, j / kChunks,
+                                x.u * kTileRows, bar(kBarFull + s));
+                }
+                __syncwarp();
+            }
+        }
+        // drain: store what is left, then let every store finish
+        while (ok && ist < it) {
+            if (updated(ist, true) < 0) ok = false;
+            else issue_store();
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+        if (*abort_flag) {
+            const uint64_t t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+        }
+    } else if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
         uint32_t it = 0;
         Unit x;
@@ -531,8 +685,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 // an epilogue thread then owns TP ADJACENT value rows, one per tile)
                 const int row = x.u * kTileRows;                      // row-group in the [units*128][TP][d_k] view of S0
                 for (int c = 0; c < kChunks; ++c, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
+                    const int s = it % NS;
+                    const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
                     if (lane == 0) {
                         mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
@@ -551,7 +705,6 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
         uint32_t it = 0, unit_seq = 0;
-        int pending_slot = -1;                                   // fused: slot whose store may still be reading it
         Unit x;
         bool ok = true;
         const uint32_t bop = sbase + kOffBop, stage = sbase + kOffStage;
@@ -589,8 +742,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             const uint32_t idm = make_idesc(2 * x.npad);
             for (int t = 0; t < TP && ok; ++t) {
                 for (int c = 0; c < kChunks; ++c, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
+                    const int s = it % NS;
+                    const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(4, bar((FUSED ? kBarUpd : kBarFull) + s), ph))) break;
                     tc_fence_after();
                     if (lane == 0) {
@@ -600,23 +753,6 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                             mma_tf32(acc + t * kAccCols, make_desc(sa + k * 32),
                                      make_desc(bop + c * kBopChunkBytes + k * 32), idm, (c | k) != 0);
                         mma_commit(bar(kBarEmpty + s));
-                        if (FUSED) {
-                            // send the advanced slice back to HBM; a slot is released one store later,
-                            // when its own store has certainly finished reading it
-                            if (x.a > 0) {
-                                tma_store_3d(&s0_map, c * kChunkK, t, x.u * kTileRows, sa);
-                                tma_store_wait_read<1>();
-                                if (pending_slot >= 0) mbar_arrive(bar(kBarEmpty + pending_slot));
-                                pending_slot = s;
-                            } else {
-                                if (pending_slot >= 0) {
-                                    tma_store_wait_read<0>();
-                                    mbar_arrive(bar(kBarEmpty + pending_slot));
-                                    pending_slot = -1;
-                                }
-                                mbar_arrive(bar(kBarEmpty + s));
-                            }
-                        }
                     }
                     __syncwarp();
                 }
@@ -629,13 +765,6 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (have) ok = issue_gram(unit_seq, x.npad);
         }
         PROF_STORE()
-        if (FUSED && lane == 0) {
-            if (pending_slot >= 0) {
-                tma_store_wait_read<0>();
-                mbar_arrive(bar(kBarEmpty + pending_slot));
-            }
-            tma_store_wait_all();
-        }
         // everything this warp issued must have completed before TMEM is released
         if (lane == 0) mma_commit(bar(kBarDrain));
         __syncwarp();
@@ -975,87 +1104,36 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         // split into a TF32 head and tail (two MMAs), so the products carry fp32 accuracy and the
         // accumulation is fp32.  The cost does not depend on A and the only shared-memory round
         // trip per batch of rows is the slice itself.
-        // Lane l keeps the index and the gate of path node l & 7; the others get them by shuffle.
-        // Everything global is fetched one unit (keys, gates) or one tile (u) ahead, and the node
-        // indices are re-read only when the sequence changes: a load whose address depends on
-        // another load costs this role a full memory round trip under a saturated HBM.
+        // The u rows and keys of the path are staged in shared memory by the TMA producer (double
+        // buffered by unit); the gates are fetched here, one unit ahead, lane l keeping the gate
+        // of path node l & 7.  Nothing on this role's path waits on a global load issued in the
+        // same unit: under a saturated HBM such a wait costs microseconds.
         const int ut = threadIdx.x - kThreads;
         const int uw = ut >> 5;                                  // warp of the role
         const int g = lane >> 2, t4 = lane & 3;                  // MMA fragment coordinates
         const int li = lane & 7;
         constexpr int kRowsPerWarp = kTileRows / kUpdWarps, kMT = kRowsPerWarp / 16;
         const int rowbase = uw * kRowsPerWarp;
-        constexpr int kKeyStride = kDK * 2 + 16;                 // bytes per staged key (bank-conflict padding)
-        constexpr int kKeyBuf = kMaxDepth * kKeyStride;
-        constexpr int kKeyPieces = kMaxDepth * 16 / kUpdThreads; // 16-byte pieces each thread copies per unit
-        int node_c = 0, node_n = 0, grp_n = -1;
         float alpha_c = 1.f, alpha_n = 1.f;
-        float wn[kMT][4];
-#pragma unroll
-        for (int m = 0; m < kMT; ++m)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) wn[m][e] = 0.f;
-        auto fetch_unit = [&](const Unit &y, int buf) {
+        auto fetch_alpha = [&](const Unit &y) {
             if (y.a == 0) return;
-            if (y.b < kWalkSeqs) {
-                node_n = reinterpret_cast<const int32_t *>(smem + kOffWalk + kWalkPBase)[y.b] +
-                         int(smem[kOffWalk + kWalkPNode + y.b * kMaxDepth + li]);
-            } else if (y.grp != grp_n) {
-                grp_n = y.grp;
-                node_n = __ldg(p.ws.pend + y.b * kPendWords + 9) + (li < y.a ? __ldg(p.ws.pend + y.b * kPendWords + 1 + li) : 0);
-            }
-            alpha_n = li < y.a ? __ldg(p.palpha + (size_t(y.l) * p.Tp + node_n) * p.H + y.h) : 1.f;
-#pragma unroll
-            for (int q = 0; q < kKeyPieces; ++q) {
-                const int piece = ut * kKeyPieces + q;           // 0..127: node piece >> 4, 16-byte piece & 15
-                const int kn = __shfl_sync(0xffffffffu, node_n, piece >> 4);
-                if ((piece >> 4) < y.a) {
-                    const __nv_bfloat16 *src = p.pk + ((size_t(y.l) * p.Tp + kn) * p.H + y.h) * kDK + (piece & 15) * 8;
-                    cp_async_16(sbase + kOffPendK + buf * kKeyBuf + (piece >> 4) * kKeyStride + (piece & 15) * 16, src);
-                }
-            }
-        };
-        // u of the pending nodes in A-fragment order: [m][0..3] = (row g, node t4), (row g + 8, node t4),
-        // (row g, node t4 + 4), (row g + 8, node t4 + 4) of m-tile m; zero past the end of the path
-        auto fetch_tile = [&](const Unit &y, int t, int node_reg) {
-            if (y.a == 0) return;
-            const int n0 = __shfl_sync(0xffffffffu, node_reg, t4), n1 = __shfl_sync(0xffffffffu, node_reg, t4 + 4);
-            const float *u0 = p.pu + ((size_t(y.l) * p.Tp + n0) * p.H + y.h) * p.DV + t;
-            const float *u1 = p.pu + ((size_t(y.l) * p.Tp + n1) * p.H + y.h) * p.DV + t;
-#pragma unroll
-            for (int m = 0; m < kMT; ++m) {
-                const int r0 = (rowbase + 16 * m + g) * TP, r1 = r0 + 8 * TP;
-                wn[m][0] = t4 < y.a ? __ldg(u0 + r0) : 0.f;
-                wn[m][1] = t4 < y.a ? __ldg(u0 + r1) : 0.f;
-                wn[m][2] = t4 + 4 < y.a ? __ldg(u1 + r0) : 0.f;
-                wn[m][3] = t4 + 4 < y.a ? __ldg(u1 + r1) : 0.f;
-            }
+            const int node = y.b < kWalkSeqs
+                ? reinterpret_cast<const int32_t *>(smem + kOffWalk + kWalkPBase)[y.b] +
+                      int(smem[kOffWalk + kWalkPNode + y.b * kMaxDepth + li])
+                : __ldg(p.ws.pend + y.b * kPendWords + 9) + (li < y.a ? __ldg(p.ws.pend + y.b * kPendWords + 1 + li) : 0);
+            alpha_n = li < y.a ? __ldg(p.palpha + (size_t(y.l) * p.Tp + node) * p.H + y.h) : 1.f;
         };
 
-        uint32_t it = 0, sync_no = 0, useq = 0;
+        uint32_t it = 0, pseq = 0;
         Unit x, nx;
         bool ok = true;
         bool have = first_unit(walk, x);
-        if (have) {
-            fetch_unit(x, 0);
-            node_c = node_n; alpha_c = alpha_n;
-            fetch_tile(x, 0, node_c);
-        }
+        if (have) { fetch_alpha(x); alpha_c = alpha_n; }
         PROF_DECL
-        auto group_sync = [&]() -> bool {
-            mbar_arrive(bar(kBarUpdSync));
-            const bool r = wait_fast(bar(kBarUpdSync), sync_no & 1, abort_flag);
-            ++sync_no;
-            return r;
-        };
-        for (; have && ok; ++useq) {
+        while (have && ok) {
             const int A = x.a;
-            const int buf = useq & 1;
+            const int pb = pseq & 1;
             PROF_MARK()
-            // this thread's key pieces of unit x have landed; after the rendezvous everybody's are
-            // visible and everybody has left the previous unit (whose key buffer is refilled below)
-            cp_async_wait_all();
-            if (!(ok = group_sync())) break;
             // my_ratio = product of alpha over the path nodes after node li; gA over all of them
             float my_ratio = 1.f, gA = 1.f;
 #pragma unroll
@@ -1070,29 +1148,35 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             PROF_SEG(1)
             nx = x;
             const bool have_next = next_unit(walk, nx);
-            if (have_next) fetch_unit(nx, buf ^ 1);
+            if (have_next) fetch_alpha(nx);
             PROF_SEG(2)
+            // the staged u rows and keys of this unit have landed
+            if (A > 0 && !(ok = WAIT(3, bar(kBarPendFull + pb), (pseq >> 1) & 1))) break;
+            const float *ub = reinterpret_cast<const float *>(smem + kOffPendU + pb * kPendUBuf);
             for (int t = 0; t < TP && ok; ++t) {
-                // A fragments of this tile: W = ratio * u
+                // A fragments of this tile, W = ratio * u: [m][0..3] = (row g, node t4), (row g + 8, node t4),
+                // (row g, node t4 + 4), (row g + 8, node t4 + 4) of m-tile m; zero past the end of the path
                 float w[kMT][4];
 #pragma unroll
                 for (int m = 0; m < kMT; ++m) {
-                    w[m][0] = ratio0 * wn[m][0]; w[m][1] = ratio0 * wn[m][1];
-                    w[m][2] = ratio1 * wn[m][2]; w[m][3] = ratio1 * wn[m][3];
+                    const int r0 = (rowbase + 16 * m + g) * TP + t, r1 = r0 + 8 * TP;
+                    const float *u0 = ub + t4 * (kPendUStride / 4), *u1 = ub + (t4 + 4) * (kPendUStride / 4);
+                    const float x0 = u0[r0], x1 = u0[r1], x2 = u1[r0], x3 = u1[r1];
+                    w[m][0] = t4 < A ? ratio0 * x0 : 0.f;
+                    w[m][1] = t4 < A ? ratio0 * x1 : 0.f;
+                    w[m][2] = t4 + 4 < A ? ratio1 * x2 : 0.f;
+                    w[m][3] = t4 + 4 < A ? ratio1 * x3 : 0.f;
                 }
-                PROF_SEG(3)
-                if (t + 1 < TP) fetch_tile(x, t + 1, node_c);
-                else if (have_next) fetch_tile(nx, 0, node_n);
                 PROF_SEG(4)
                 for (int c = 0; c < kChunks; ++c, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
+                    const int s = it % NS;
+                    const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarFull + s), ph))) break;
                     PROF_MARK()
                     if (A > 0) {
                         uint8_t *slot = smem + kOffRing + s * kStageBytes;
                         // B fragments: keys t4 and t4 + 4 at column 8 n + g of this chunk
-                        const uint8_t *kb = smem + kOffPendK + buf * kKeyBuf + (c * kChunkK + g) * 2;
+                        const uint8_t *kb = smem + kOffPendK + pb * kKeyBuf + (c * kChunkK + g) * 2;
                         uint32_t b0[4], b1[4];
 #pragma unroll
                         for (int n = 0; n < 4; ++n) {
@@ -1152,13 +1236,13 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     PROF_SEG(6)
                 }
             }
+            // the staged rows may be refilled
+            if (A > 0) { mbar_arrive(bar(kBarPendFree + pb)); ++pseq; }
             x = nx;
             have = have_next;
-            node_c = node_n;
             alpha_c = alpha_n;
         }
         PROF_STORE()
-        cp_async_wait_all();
     }
 
     tc_fence_before();
