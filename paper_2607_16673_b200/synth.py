@@ -92,6 +92,37 @@ def beam_tree_parent(top_k: int, depth: int, n_nodes: int, rng: np.random.Genera
     return np.asarray(parent, dtype=np.int32)
 
 
+def proposal_tree_parent(top_k: int, depth: int, n_nodes: int, rng: np.random.Generator,
+                         max_depth: int = 16) -> np.ndarray:
+    """Proposal tree with the metadata the paper reports per shape (top-k, configured depth,
+    total nodes): ``n_nodes`` spread as evenly as possible over ``min(depth, max_depth)`` levels,
+    a node having at most ``top_k`` children, parents drawn at random among the previous
+    level's nodes that still have room.  Level order, so topological and ancestor-closed."""
+    levels = min(depth, max_depth, n_nodes)
+    width = [n_nodes // levels + (1 if i < n_nodes % levels else 0) for i in range(levels)]
+    # a level can hold at most top_k children per node of the level above it
+    cap = top_k
+    for i in range(levels):
+        if width[i] > cap:
+            if i + 1 < levels:
+                width[i + 1] += width[i] - cap
+            width[i] = cap
+        cap = width[i] * top_k
+    parent: List[int] = []
+    prev: List[int] = [-1]
+    for w in width:
+        room = {p: top_k for p in prev}
+        cur: List[int] = []
+        for j in range(w):
+            cands = [p for p in prev if room[p] > 0]
+            p = cands[0] if j == 0 else cands[int(rng.integers(len(cands)))]
+            room[p] -= 1
+            parent.append(p)
+            cur.append(len(parent) - 1)
+        prev = cur
+    return np.asarray(parent, dtype=np.int32)
+
+
 # ----------------------------------------------------------------------------
 # problem container
 # ----------------------------------------------------------------------------
