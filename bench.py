@@ -37,6 +37,9 @@ WORKLOADS = {
     "cfg5": (24, 128, 16, 128, 256, "128 seq x 24 layers x 16 heads, d_k=128 d_v=256; 64 seq with 8-token chains + "
                                     "64 seq with 64-node trees (depth<=8)"),
     "cfg4": (24, 32, 16, 128, 256, "32 seq x 24 layers x 16 heads, d_k=128 d_v=256; ragged trees of 8..64 nodes (depth<=8)"),
+    # the paper's target shape (h_v = 8, d_k = d_v = 256, 24 layers) served in a batch
+    "paper256": (24, 64, 8, 256, 256, "64 seq x 24 layers x 8 heads, d_k=d_v=256 (the paper's target shape); 32 seq with "
+                                      "8-token chains + 32 seq with top-4 proposal trees of 16..32 nodes (depth 4..8)"),
 }
 POOL = 3            # independent draft inputs rotated over the steps ("fresh draft factors each round")
 
@@ -68,6 +71,10 @@ def host_round_inputs(name: str, B: int, seed: int):
     rng = np.random.default_rng(seed)
     if name == "cfg5":
         parents = synth.mixed_chain_tree_batch(rng, B, 8, 64, 8)
+    elif name == "paper256":
+        parents = [synth.chain_parent(8) for _ in range(B // 2)]
+        parents += [synth.proposal_tree_parent(4, int(rng.integers(4, 9)), int(rng.integers(16, 33)), rng, 8)
+                    for _ in range(B - B // 2)]
     else:
         parents = synth.ragged_tree_batch(rng, B, 8, 64, 8)
     sizes = [len(p) for p in parents]
@@ -212,7 +219,7 @@ def run_speca(args):
     L, B, H, dk, dv, desc = WORKLOADS[args.workload]
     L = args.layers or L
     B = args.batch or B
-    dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, args.route)
+    dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64 if dk <= 128 else 32, args.route)
     stream = torch.cuda.current_stream()
 
     # --- inputs resident in HBM -------------------------------------------------
@@ -345,7 +352,7 @@ def run_speca(args):
         "config": {"workload": f"{args.workload}: {desc}", "n_layers": L, "batch_per_gpu": B, "heads": H,
                    "d_k": dk, "d_v": dv, "nodes_per_step_per_gpu": [p["T"] for p in pool],
                    "mean_accepted_len": float(np.mean([p["path_len"].mean() for p in pool])),
-                   "input_pool": POOL, "l2": "inputs larger than L2 (state 6.4 GB, records 1.8 GB per round at full size)",
+                   "input_pool": POOL, "l2": f"inputs larger than L2 (state {L * B * H * dk * dv * 4 / 1e9:.1f} GB)",
                    "route": args.route, "parallelism": f"dp{world} (sequences partitioned, no collective)"},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get(dom) if args.workload == "cfg5" and not args.layers and not args.batch else None,
@@ -495,6 +502,10 @@ def oracle_sample_problem(workload: str, H: int, dk: int, dv: int, n_units: int,
     rng = np.random.default_rng(seed)
     if workload == "cfg5":
         parents = synth.mixed_chain_tree_batch(rng, n_units, 8, 64, 8)
+    elif workload == "paper256":
+        parents = [synth.chain_parent(8) for _ in range(n_units // 2)]
+        parents += [synth.proposal_tree_parent(4, int(rng.integers(4, 9)), int(rng.integers(16, 33)), rng, 8)
+                    for _ in range(n_units - n_units // 2)]
     else:
         parents = synth.ragged_tree_batch(rng, n_units, 8, 64, 8)
     return synth.make_problem(seed, 1, 1, dk, dv, parents)
@@ -589,7 +600,9 @@ def run_paper_shapes(args):
         par = synth.proposal_tree_parent(top_k, depth, nodes, rng, 16)      # the library takes depth <= 16
         prob = synth.make_problem(77 + nodes + top_k, L, H, dk, dv, [par], max_depth=16)
         n = len(par)
-        dims = speca.Dims(L, 1, H, dk, dv, 1.0, 16, 64, args.route)
+        tree_depth = int(synth.depth_of(par).max())
+        md = 8 if tree_depth <= 8 else 16            # depth <= 8 and <= 32 nodes: the tensor-core route applies
+        dims = speca.Dims(L, 1, H, dk, dv, 1.0, md, 32, args.route)
         S = [t(prob.S0) + 0 for _ in range(COPIES)]
         q, k, v, al, be = bf(prob.q), bf(prob.k), bf(prob.v), t(prob.alpha), t(prob.beta)
         offs, parent = t(prob.node_offsets), t(prob.parent)
@@ -605,7 +618,7 @@ def run_paper_shapes(args):
         idx = np.concatenate(paths)
         offs_r = np.concatenate([[0], np.cumsum([len(p) for p in paths])]).astype(np.int32)
         Br, Tr = len(paths), int(offs_r[-1])
-        dims_r = speca.Dims(L, Br, H, dk, dv, 1.0, 16, 64, args.route)
+        dims_r = speca.Dims(L, Br, H, dk, dv, 1.0, md, 32, args.route)
         Sr = [S[c].expand(L, Br, H, dv, dk).contiguous() for c in range(2)]
         take = lambda x: x[:, t(idx).long()].contiguous()
         qr, kr, vr, alr, ber = take(q), take(k), take(v), take(al), take(be)
@@ -615,12 +628,12 @@ def run_paper_shapes(args):
                                                     status))
         # commit of the deepest path
         path = max(paths, key=len)[:8]
-        pidx = torch.full((1, 16), -1, dtype=torch.int32, device=dev)
+        pidx = torch.full((1, md), -1, dtype=torch.int32, device=dev)
         pidx[0, :len(path)] = t(np.asarray(path, np.int32))
         plen = torch.tensor([len(path)], dtype=torch.int32, device=dev)
         ms_commit = timed(lambda i: speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent, pidx, plen, status))
         assert int(status.item()) == 0
-        rows.append({"top_k": top_k, "config_depth": depth, "nodes": n, "tree_depth": int(synth.depth_of(par).max()),
+        rows.append({"top_k": top_k, "config_depth": depth, "nodes": n, "tree_depth": tree_depth,
                      "leaves": Br, "replayed_tokens": Tr, "verify_tree_ms": ms_tree, "r2l_replay_ms": ms_r2l,
                      "tree_vs_r2l": ms_r2l / ms_tree, "commit_ms": ms_commit, "accepted_len": len(path),
                      "token_layers_per_s": n * L / ((ms_tree + ms_commit) * 1e-3)})

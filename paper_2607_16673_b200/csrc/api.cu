@@ -71,7 +71,7 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
         rc = cuda_rc(launch_plan(p, st));
         if (rc != SPECA_OK) return rc;
     }
-    if (factorize) return cuda_rc(launch_verify_factorized(p, false, st));
+    if (factorize) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, st));
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 
@@ -247,7 +247,7 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k
 
     // One pass over the state when the tensor-core route applies and the previous verification
     // left its u; otherwise the two kernels run back to back on the stream (same results).
-    const bool one_pass = have_commit && total_nodes > 0 && u_prev_or_null != nullptr && factorized_supported(dims) &&
+    const bool one_pass = have_commit && total_nodes > 0 && u_prev_or_null != nullptr && factorized_fused_supported(dims) &&
                           dims->route != SPECA_ROUTE_SERIAL;
     if (!one_pass) {
         if (have_commit) {
@@ -288,7 +288,7 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k
     if (rc != SPECA_OK) return rc;
     rc = cuda_rc(launch_pending_check(p, 8, st));
     if (rc != SPECA_OK) return rc;
-    return cuda_rc(launch_verify_factorized(p, true, st));
+    return cuda_rc(launch_verify_factorized(p, dims->d_k, true, st));
 }
 
 }  // extern "C"

@@ -479,8 +479,10 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
     }
 }
 
-// TP = value tiles per unit (d_v / 128): 1 or 2.  FUSED adds the state-update role.
-template <int TP, bool FUSED>
+// TP = value tiles per unit (d_v / 128): 1 or 2.  FUSED adds the state-update role (d_k = 128 only).
+// DK = key width, 128 or 256.  The operand buffers have a fixed size, so the wider key halves
+// the number of [K;Q] rows they hold: up to 64 nodes per sequence at d_k = 128, 32 at d_k = 256.
+template <int TP, bool FUSED, int DK = kDK>
 __global__ void __launch_bounds__(FUSED ? kThreadsFused : kThreads, 1)
 verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
@@ -543,6 +545,14 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int NS = FUSED ? kStagesFused : kStages;            // ring depth in use
+    static_assert(DK == 128 || DK == 256, "key width");
+    static_assert(!FUSED || DK == kDK, "the fused kernel is built for d_k = 128");
+    constexpr int NC = DK / kChunkK;                              // K-chunks (state slices) per tile
+    constexpr int BROWS = DK == 128 ? kBopRows : kBopRows / 2;    // [K;Q] rows the operand buffers hold
+    constexpr int BCB = BROWS * 128;                              // bytes of one K-chunk region of the fp32 operand
+    constexpr int SC = DK / 64;                                   // 64-column chunks of the staged bf16 rows
+    constexpr int SCB = BROWS * 128;                              // bytes of one such chunk
+    static_assert(NC * BCB == kChunks * kBopChunkBytes && SC * SCB == 2 * kStageChunkBytes, "operand buffers keep their size");
     UnitWalk walk;
     walk.HG = fp.heads_per_group; walk.gpl = p.H / fp.heads_per_group;
     walk.n_groups = int(fp.n_units / fp.heads_per_group);
@@ -684,7 +694,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 // tile t of a unit holds its value rows t, t + TP, t + 2 TP, ... (interleaved tiles:
                 // an epilogue thread then owns TP ADJACENT value rows, one per tile)
                 const int row = x.u * kTileRows;                      // row-group in the [units*128][TP][d_k] view of S0
-                for (int c = 0; c < kChunks; ++c, ++it) {
+                for (int c = 0; c < NC; ++c, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
@@ -720,10 +730,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (lane == 0) {
                 const uint32_t idg = make_idesc_bf16(npad);
 #pragma unroll
-                for (int c = 0; c < 2; ++c)
+                for (int c = 0; c < SC; ++c)
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const uint64_t d = make_desc(stage + c * kStageChunkBytes + k * 32);
+                        const uint64_t d = make_desc(stage + c * SCB + k * 32);
                         mma_bf16(tmem_base + pr * kPairCols, d, d, idg, (c | k) != 0);
                     }
                 mma_commit(bar(kBarGramFull));
@@ -741,7 +751,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             tc_fence_after();
             const uint32_t idm = make_idesc(2 * x.npad);
             for (int t = 0; t < TP && ok; ++t) {
-                for (int c = 0; c < kChunks; ++c, ++it) {
+                for (int c = 0; c < NC; ++c, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(4, bar((FUSED ? kBarUpd : kBarFull) + s), ph))) break;
@@ -751,7 +761,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             mma_tf32(acc + t * kAccCols, make_desc(sa + k * 32),
-                                     make_desc(bop + c * kBopChunkBytes + k * 32), idm, (c | k) != 0);
+                                     make_desc(bop + c * BCB + k * 32), idm, (c | k) != 0);
                         mma_commit(bar(kBarEmpty + s));
                     }
                     __syncwarp();
@@ -781,16 +791,16 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         // staging buffer laid out as a bf16 K-major 128-byte-swizzled operand: rows [0, npad) keys,
         // [npad, 2 npad) queries.  The Gram MMA reads it directly; the conversion below gathers
         // its rows in depth-first order into the fp32 operand of the state MMAs.
-        // This thread converts, for operand rows r = sub, sub + 8, ..., the 16-byte piece seg of
+        // This thread converts, for operand rows r = sub, sub + RSTEP, ..., the 16-byte piece seg of
         // the row (bf16 columns 8 seg .. 8 seg + 7).
         const uint32_t stage = sbase + kOffStage;
-        const int sub = tid >> 4, seg = tid & 15;
+        constexpr int PPR = DK / 8;                              // 16-byte bf16 pieces per row
+        constexpr int RSTEP = kPrepThreads / PPR;                // rows converted per pass: 8 (d_k 128) or 4 (d_k 256)
+        const int sub = tid / PPR, seg = tid % PPR;
         // staging piece of node nd: chunk (seg >> 3) of 64 bf16, 16-byte slot (seg & 7) ^ (nd & 7)
-        const uint32_t stage_chunk = uint32_t((seg >> 3) * kStageChunkBytes);
-        // fp32 operand: floats 8 seg .. 8 seg + 7 -> chunk seg >> 2, 16-byte slots 2 (seg & 3), +1;
-        // r & 7 == sub for every handled row
-        const uint32_t bop_off0 = uint32_t((seg >> 2) * kBopChunkBytes + sub * 128 + (((2 * (seg & 3)) ^ sub) << 4));
-        const uint32_t bop_off1 = uint32_t((seg >> 2) * kBopChunkBytes + sub * 128 + (((2 * (seg & 3) + 1) ^ sub) << 4));
+        const uint32_t stage_chunk = uint32_t((seg >> 3) * SCB);
+        // fp32 operand: floats 8 seg .. 8 seg + 7 -> chunk seg >> 2, 16-byte slots 2 (seg & 3), +1 (swizzled by r & 7)
+        const uint32_t bop_chunk = uint32_t((seg >> 2) * BCB);
 
         float my_alpha = 0.f, my_beta = 0.f;
         unsigned long long node_lo = ~0ull, node_hi = ~0ull;   // node at the position of each handled row (0xff = none)
@@ -802,11 +812,11 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (tid == 0) {
                 const int m = (x.npad >> 4) - 1;             // box height 16 (m + 1)
                 const int z = x.l * p.T + x.base;
-                mbar_arrive_expect_tx(bar(kBarStageReady), uint32_t(4 * x.npad * 128));
+                mbar_arrive_expect_tx(bar(kBarStageReady), uint32_t(4 * x.npad * DK));
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    tma_load_3d(stage + c * kStageChunkBytes, &kq.k[m], c * 64, x.h, z, bar(kBarStageReady));
-                    tma_load_3d(stage + c * kStageChunkBytes + x.npad * 128, &kq.q[m], c * 64, x.h, z, bar(kBarStageReady));
+                for (int c = 0; c < SC; ++c) {
+                    tma_load_3d(stage + c * SCB, &kq.k[m], c * 64, x.h, z, bar(kBarStageReady));
+                    tma_load_3d(stage + c * SCB + x.npad * 128, &kq.q[m], c * 64, x.h, z, bar(kBarStageReady));
                 }
             }
             if (x.grp != topo_grp) {
@@ -814,7 +824,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 node_lo = node_hi = 0ull;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const int r = 8 * i + sub;
+                    const int r = RSTEP * i + sub;
                     const int pos = r < x.npad ? r : r - x.npad;
                     const unsigned long long nd =
                         (r < 2 * x.npad && pos < x.n) ? (unsigned long long)(__ldg(p.ws.plan + x.base + pos) & 0xff) : 0xffull;
@@ -853,11 +863,14 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (!(ok = WAIT(2, bar(kBarStageReady), unit_seq & 1))) break;
             {
                 // bf16 -> fp32 (exact): operand row r (depth-first position) <- staged row of its node
-                const int iters = x.npad >> 2;               // 2 npad / 8
-                const int nk = x.npad >> 3;                  // rows [0, npad) keys, then queries
-                uint8_t *dst = smem + kOffBop;
+                const int iters = 2 * x.npad / RSTEP;
+                const int nk = x.npad / RSTEP;               // rows [0, npad) keys, then queries
 #pragma unroll 4
-                for (int i = 0; i < iters; ++i, dst += 1024) {
+                for (int i = 0; i < iters; ++i) {
+                    const int r = RSTEP * i + sub;
+                    uint8_t *dst = smem + kOffBop + bop_chunk + r * 128;
+                    const uint32_t bop_off0 = uint32_t(((2 * (seg & 3)) ^ (r & 7)) << 4);
+                    const uint32_t bop_off1 = uint32_t(((2 * (seg & 3) + 1) ^ (r & 7)) << 4);
                     const int nd = int(((i < 8 ? cur_lo : cur_hi) >> (8 * (i & 7))) & 0xffull);
                     uint4 w = make_uint4(0u, 0u, 0u, 0u);
                     if (nd != 0xff) {
@@ -1275,19 +1288,22 @@ EncodeTiledFn encode_tiled_fn()
 
 bool factorized_supported(const speca_dims *d)
 {
-    return d->d_k == kDK && (d->d_v == kTileRows || d->d_v == 2 * kTileRows) && d->max_nodes <= kMaxNodes &&
-           d->max_depth <= kMaxDepth;
+    const bool keys = (d->d_k == kDK && d->max_nodes <= kMaxNodes) || (d->d_k == 2 * kDK && d->max_nodes <= kMaxNodes / 2);
+    return keys && (d->d_v == kTileRows || d->d_v == 2 * kTileRows) && d->max_depth <= kMaxDepth;
 }
 
-int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st)
+bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d) && d->d_k == kDK; }
+
+int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st)
 {
+    if ((d_k != kDK && d_k != 2 * kDK) || (fused && d_k != kDK)) return int(cudaErrorInvalidValue);
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return int(cudaErrorNotSupported);
     const long n_units = long(p.L) * p.B * p.H;
     CUtensorMap map;
     const int tiles = p.DV / kTileRows;
-    const cuuint64_t gdim[3] = {cuuint64_t(kDK), cuuint64_t(tiles), cuuint64_t(n_units) * kTileRows};
-    const cuuint64_t gstride[2] = {cuuint64_t(kDK) * sizeof(float), cuuint64_t(tiles) * kDK * sizeof(float)};
+    const cuuint64_t gdim[3] = {cuuint64_t(d_k), cuuint64_t(tiles), cuuint64_t(n_units) * kTileRows};
+    const cuuint64_t gstride[2] = {cuuint64_t(d_k) * sizeof(float), cuuint64_t(tiles) * d_k * sizeof(float)};
     const cuuint32_t box[3] = {kChunkK, 1, kTileRows};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(p.S0), gdim, gstride, box, estr,
@@ -1297,8 +1313,8 @@ int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st)
 
     KQMaps kq;
     {
-        const cuuint64_t gd[3] = {cuuint64_t(kDK), cuuint64_t(p.H), cuuint64_t(p.L) * cuuint64_t(p.T)};
-        const cuuint64_t gs[2] = {cuuint64_t(kDK) * 2, cuuint64_t(p.H) * kDK * 2};
+        const cuuint64_t gd[3] = {cuuint64_t(d_k), cuuint64_t(p.H), cuuint64_t(p.L) * cuuint64_t(p.T)};
+        const cuuint64_t gs[2] = {cuuint64_t(d_k) * 2, cuuint64_t(p.H) * d_k * 2};
         const cuuint32_t es[3] = {1, 1, 1};
         for (int m = 0; m < 4; ++m) {
             const cuuint32_t bx[3] = {64, 1, cuuint32_t(16 * (m + 1))};
@@ -1328,32 +1344,39 @@ int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st)
     }
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(verify_factorized_kernel<1, false>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(verify_factorized_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(verify_factorized_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(verify_factorized_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemBytes);
-        if (e != cudaSuccess) return int(e);
+        const void *kernels[] = {
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 128>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 128>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 128>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 128>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256>)};
+        for (const void *k : kernels) {
+            cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            if (e != cudaSuccess) return int(e);
+        }
         attr_set = true;
     }
     FParams fp;
     fp.p = p;
     fp.n_units = n_units;
-    fp.heads_per_group = (p.H % 4 == 0) ? 4 : (p.H % 2 == 0 ? 2 : 1);
+    // consecutive heads of one (layer, sequence) a CTA takes together: as many as divide H while
+    // every SM still gets a group
+    fp.heads_per_group = 1;
+    for (int hg = 4; hg > 1; hg >>= 1)
+        if (p.H % hg == 0 && n_units / hg >= sm_count) { fp.heads_per_group = hg; break; }
     const long n_groups = n_units / fp.heads_per_group;
     const int grid = int(n_groups < sm_count ? n_groups : sm_count);
+    const bool one_tile = p.DV == kTileRows;
     if (fused) {
-        if (p.DV == kTileRows) verify_factorized_kernel<1, true><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, true><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+        if (one_tile) verify_factorized_kernel<1, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+    } else if (d_k == kDK) {
+        if (one_tile) verify_factorized_kernel<1, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
     } else {
-        if (p.DV == kTileRows) verify_factorized_kernel<1, false><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, false><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        if (one_tile) verify_factorized_kernel<1, false, 256><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, false, 256><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
     }
     return int(cudaGetLastError());
 }

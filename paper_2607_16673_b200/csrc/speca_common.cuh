@@ -96,7 +96,8 @@ int launch_decode(const Params &p, int d_k, cudaStream_t st);
 int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
 int launch_commit(const Params &p, int d_k, cudaStream_t st);
 bool factorized_supported(const speca_dims *d);
-int launch_verify_factorized(const Params &p, bool fused, cudaStream_t st);
+bool factorized_fused_supported(const speca_dims *d);
+int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st);
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
 int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
                   const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,

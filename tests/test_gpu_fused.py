@@ -114,6 +114,15 @@ def test_fused_shapes_outside_the_tensor_core_route():
     assert rel_err(cpu(S), S_ref) <= TOL_FP32
 
 
+def test_fused_key_width_256_takes_the_two_kernel_path():
+    """d_k = 256 is on the tensor-core route for verification but not for the single-pass kernel."""
+    rng = np.random.default_rng(13)
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(45, 2, 8, 256, 256, synth.ragged_tree_batch(rng, 3, 4, 32, 8),
+                                               synth.ragged_tree_batch(rng, 3, 4, 32, 8), speca.ROUTE_AUTO, max_nodes=32)
+    assert rel_err(cpu(d2.o), o_ref) <= TOL
+    assert rel_err(cpu(S), S_ref) <= TOL_FP32
+
+
 def test_nothing_pending_and_nothing_to_verify():
     rng = np.random.default_rng(8)
     prob = synth.make_problem(51, 2, 4, 128, 256, synth.ragged_tree_batch(rng, 3, 8, 30, 8))

@@ -387,3 +387,39 @@ def test_factorized_faults_skip_the_sequence():
     assert np.all(np.isnan(o[:, s1:e1]))
     keep = np.r_[0:s1, e1:prob.T]
     assert rel_err(o[:, keep], good[:, keep]) <= TOL
+
+
+@pytest.mark.parametrize("d_v", [128, 256])
+def test_factorized_key_width_256(d_v):
+    """The paper's target shape (d_k = 256): the tensor-core route takes up to 32 nodes per sequence."""
+    rng = np.random.default_rng(970 + d_v)
+    forest = np.array([-1, -1, 0, -1, 1, 1, 2, 3, 3, 6], np.int32)
+    parents = [np.zeros(0, np.int32), synth.chain_parent(1), forest, synth.chain_parent(8),
+               synth.random_tree_parent(32, 8, 4, rng), synth.proposal_tree_parent(4, 4, 32, rng),
+               synth.random_tree_parent(17, 8, 2, rng), synth.proposal_tree_parent(4, 4, 16, rng),
+               synth.random_tree_parent(29, 5, 4, rng)]
+    prob = synth.make_problem(971 + d_v, 3, 8, 256, d_v, parents, name=f"fact-dk256-{d_v}")
+    dp, ref = check_verify(prob, speca.ROUTE_FACTORIZED, want_u=True, max_nodes=32)
+    ds = DevProblem(prob, route=speca.ROUTE_SERIAL, want_u=True, max_nodes=32)
+    ds.verify_tree()
+    assert rel_err(cpu(dp.o), cpu(ds.o)) <= TOL and rel_err(cpu(dp.u), cpu(ds.u)) <= TOL
+    # accept + commit on the same records (commit is the fp32 kernel whatever verified)
+    dp.accept()
+    pi, pl, _ = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                     prob.root_target_tok, prob.max_depth)
+    assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+    dp.commit()
+    assert rel_err(cpu(dp.S), oracle_commit(prob, pi, pl)) <= TOL_FP32
+    # 33 nodes is one too many for this key width: refused when asked for explicitly, serial under AUTO
+    big = synth.make_problem(972, 1, 2, 256, d_v, [synth.random_tree_parent(33, 8, 4, rng)])
+    with pytest.raises(speca.SpecaError, match="unsupported"):
+        DevProblem(big, route=speca.ROUTE_FACTORIZED, max_nodes=33).verify_tree()
+    check_verify(big, speca.ROUTE_AUTO, tol=TOL_FP32, max_nodes=33)
+
+
+def test_factorized_key_width_256_batched_paper_shape():
+    """h_v = 8, d_k = d_v = 256, a batch of proposal trees (depth <= 8): every unit against the oracle."""
+    rng = np.random.default_rng(980)
+    parents = [synth.proposal_tree_parent(4, int(rng.integers(3, 9)), int(rng.integers(8, 33)), rng) for _ in range(24)]
+    prob = synth.make_problem(981, 2, 8, 256, 256, parents, name="paper-shape-batch")
+    check_verify(prob, speca.ROUTE_AUTO, max_nodes=32)
