@@ -546,13 +546,22 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 
     constexpr int NS = FUSED ? kStagesFused : kStages;            // ring depth in use
     static_assert(DK == 128 || DK == 256, "key width");
-    static_assert(!FUSED || DK == kDK, "the fused kernel is built for d_k = 128");
     constexpr int NC = DK / kChunkK;                              // K-chunks (state slices) per tile
     constexpr int BROWS = DK == 128 ? kBopRows : kBopRows / 2;    // [K;Q] rows the operand buffers hold
     constexpr int BCB = BROWS * 128;                              // bytes of one K-chunk region of the fp32 operand
     constexpr int SC = DK / 64;                                   // 64-column chunks of the staged bf16 rows
     constexpr int SCB = BROWS * 128;                              // bytes of one such chunk
     static_assert(NC * BCB == kChunks * kBopChunkBytes && SC * SCB == 2 * kStageChunkBytes, "operand buffers keep their size");
+    constexpr int MAXN = BROWS / 2;                               // nodes per sequence; also the stride of the coefficient buffers
+    // Fused kernel: staged bf16 keys of the pending path, two buffers of 8 padded rows.  At d_k = 128 both
+    // sit in their own region; at d_k = 256 a buffer is twice as large, and the second one takes the half
+    // of the coefficient region that 32-node sequences leave unused.
+    constexpr int KSTRIDE = DK * 2 + 16, KBUF = kMaxDepth * KSTRIDE;
+    static_assert(DK == kDK ? 2 * KBUF <= kOffWalk - kOffPendK
+                            : (KBUF <= kOffWalk - kOffPendK && KBUF <= kMaxNodes * kCoefStride * 4), "pending keys do not fit");
+    auto key_buf = [](int pb) -> int {
+        return DK == kDK ? kOffPendK + pb * KBUF : (pb == 0 ? kOffPendK : kOffCoef + 2 * MAXN * kCoefStride * 4);
+    };
     UnitWalk walk;
     walk.HG = fp.heads_per_group; walk.gpl = p.H / fp.heads_per_group;
     walk.n_groups = int(fp.n_units / fp.heads_per_group);
@@ -578,7 +587,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             if (y.a == 0) return true;
             const int pb = pseq & 1;
             if (!wait_fast(bar(kBarPendFree + pb), ((pseq >> 1) & 1) ^ 1, abort_flag)) return false;
-            if (lane == 0) mbar_arrive_expect_tx(bar(kBarPendFull + pb), uint32_t(y.a) * uint32_t(p.DV * 4 + kDK * 2));
+            if (lane == 0) mbar_arrive_expect_tx(bar(kBarPendFull + pb), uint32_t(y.a) * uint32_t(p.DV * 4 + DK * 2));
             __syncwarp();
             if (lane < y.a) {
                 const int node = y.b < kWalkSeqs
@@ -588,7 +597,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 const size_t rec = (size_t(y.l) * p.Tp + node) * p.H + y.h;
                 bulk_load(sbase + kOffPendU + pb * kPendUBuf + lane * kPendUStride, p.pu + rec * p.DV, uint32_t(p.DV * 4),
                           bar(kBarPendFull + pb));
-                bulk_load(sbase + kOffPendK + pb * kKeyBuf + lane * kKeyStride, p.pk + rec * kDK, uint32_t(kDK * 2),
+                bulk_load(sbase + key_buf(pb) + lane * KSTRIDE, p.pk + rec * DK, uint32_t(DK * 2),
                           bar(kBarPendFull + pb));
             }
             ++pseq;
@@ -598,13 +607,13 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         auto issue_store = [&]() {
             if (lane == 0) {
                 if (xs.a > 0)
-                    tma_store_3d_nocommit(&s0_map, (js % kChunks) * kChunkK, js / kChunks, xs.u * kTileRows,
+                    tma_store_3d_nocommit(&s0_map, (js % NC) * kChunkK, js / NC, xs.u * kTileRows,
                                           sbase + kOffRing + (ist % NS) * kStageBytes);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
             __syncwarp();
             ++ist;
-            if (++js == TP * kChunks) { js = 0; next_unit(walk, xs); }
+            if (++js == TP * NC) { js = 0; next_unit(walk, xs); }
         };
         auto updated = [&](uint32_t i, bool blocking) -> int {   // 1 ready, 0 not yet, -1 abort
             if (xs.a == 0) return 1;
@@ -620,10 +629,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             const bool have_next = next_unit(walk, nx);
             have = have_next;
             if (lane == 0 && x.n > 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
-            for (int j = 0; j < TP * kChunks && ok; ++j, ++it) {
+            for (int j = 0; j < TP * NC && ok; ++j, ++it) {
                 // halfway through the unit the update role has left the unit before it, whose
                 // staging buffer the next unit's pending path takes
-                if (have_next && j == TP * kChunks / 2 && !(ok = stage_pending(nx))) break;
+                if (have_next && j == TP * NC / 2 && !(ok = stage_pending(nx))) break;
                 const int s = it % NS;
                 if (it >= uint32_t(NS)) {
                     // the slot's previous content (slice it - NS) must have been stored ...
@@ -663,7 +672,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 }
                 if (lane == 0) {
                     mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
-                    tma_load_3d(sbase + kOffRing + s * kStageBytes, &s0_map, (j % kChunks) * kChunkK, j / kChunks,
+                    tma_load_3d(sbase + kOffRing + s * kStageBytes, &s0_map, (j % NC) * kChunkK, j / NC,
                                 x.u * kTileRows, bar(kBarFull + s));
                 }
                 __syncwarp();
@@ -944,7 +953,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             // coefficient record of this row's node; levels that are not ancestors stay zero, rows
             // past the last node (padding up to a multiple of 16) become no-op records
             if (in_rows) {
-                float *cf = reinterpret_cast<float *>(smem + kOffCoef) + (par * kMaxNodes + pos) * kCoefStride;
+                float *cf = reinterpret_cast<float *>(smem + kOffCoef) + (par * MAXN + pos) * kCoefStride;
                 float c[kMaxDepth];
                 float ratio = my_a;
 #pragma unroll
@@ -992,7 +1001,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
         const uint32_t acc = tmem_base + grp * kPairCols + lane_addr;
-        const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * kMaxNodes * kCoefStride;
+        const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * MAXN * kCoefStride;
 
         // this group's units: unit_seq == grp (mod 2)
         Unit x;
@@ -1181,7 +1190,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     w[m][3] = t4 + 4 < A ? ratio1 * x3 : 0.f;
                 }
                 PROF_SEG(4)
-                for (int c = 0; c < kChunks; ++c, ++it) {
+                for (int c = 0; c < NC; ++c, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarFull + s), ph))) break;
@@ -1189,12 +1198,12 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     if (A > 0) {
                         uint8_t *slot = smem + kOffRing + s * kStageBytes;
                         // B fragments: keys t4 and t4 + 4 at column 8 n + g of this chunk
-                        const uint8_t *kb = smem + kOffPendK + pb * kKeyBuf + (c * kChunkK + g) * 2;
+                        const uint8_t *kb = smem + key_buf(pb) + (c * kChunkK + g) * 2;
                         uint32_t b0[4], b1[4];
 #pragma unroll
                         for (int n = 0; n < 4; ++n) {
-                            const uint32_t lo = *reinterpret_cast<const unsigned short *>(kb + t4 * kKeyStride + n * 16);
-                            const uint32_t hi = *reinterpret_cast<const unsigned short *>(kb + (t4 + 4) * kKeyStride + n * 16);
+                            const uint32_t lo = *reinterpret_cast<const unsigned short *>(kb + t4 * KSTRIDE + n * 16);
+                            const uint32_t hi = *reinterpret_cast<const unsigned short *>(kb + (t4 + 4) * KSTRIDE + n * 16);
                             b0[n] = t4 < A ? lo << 16 : 0u;
                             b1[n] = t4 + 4 < A ? hi << 16 : 0u;
                         }
@@ -1292,11 +1301,11 @@ bool factorized_supported(const speca_dims *d)
     return keys && (d->d_v == kTileRows || d->d_v == 2 * kTileRows) && d->max_depth <= kMaxDepth;
 }
 
-bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d) && d->d_k == kDK; }
+bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d); }
 
 int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st)
 {
-    if ((d_k != kDK && d_k != 2 * kDK) || (fused && d_k != kDK)) return int(cudaErrorInvalidValue);
+    if (d_k != kDK && d_k != 2 * kDK) return int(cudaErrorInvalidValue);
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return int(cudaErrorNotSupported);
     const long n_units = long(p.L) * p.B * p.H;
@@ -1350,7 +1359,9 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
             reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 128>),
             reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 128>),
             reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256>)};
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 256>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 256>)};
         for (const void *k : kernels) {
             cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
             if (e != cudaSuccess) return int(e);
@@ -1368,9 +1379,12 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
     const long n_groups = n_units / fp.heads_per_group;
     const int grid = int(n_groups < sm_count ? n_groups : sm_count);
     const bool one_tile = p.DV == kTileRows;
-    if (fused) {
+    if (fused && d_k == kDK) {
         if (one_tile) verify_factorized_kernel<1, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
         else verify_factorized_kernel<2, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+    } else if (fused) {
+        if (one_tile) verify_factorized_kernel<1, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
     } else if (d_k == kDK) {
         if (one_tile) verify_factorized_kernel<1, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
         else verify_factorized_kernel<2, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);

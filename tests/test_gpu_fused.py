@@ -114,13 +114,19 @@ def test_fused_shapes_outside_the_tensor_core_route():
     assert rel_err(cpu(S), S_ref) <= TOL_FP32
 
 
-def test_fused_key_width_256_takes_the_two_kernel_path():
-    """d_k = 256 is on the tensor-core route for verification but not for the single-pass kernel."""
-    rng = np.random.default_rng(13)
-    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(45, 2, 8, 256, 256, synth.ragged_tree_batch(rng, 3, 4, 32, 8),
-                                               synth.ragged_tree_batch(rng, 3, 4, 32, 8), speca.ROUTE_AUTO, max_nodes=32)
+@pytest.mark.parametrize("d_v", [128, 256])
+def test_fused_key_width_256(d_v):
+    """The paper's target shape on the single-pass kernel (up to 32 nodes per sequence)."""
+    rng = np.random.default_rng(13 + d_v)
+    prev = synth.ragged_tree_batch(rng, 5, 4, 32, 8) + [synth.chain_parent(8), np.zeros(0, np.int32)]
+    new = synth.ragged_tree_batch(rng, 5, 4, 32, 8) + [np.zeros(0, np.int32), synth.chain_parent(8)]
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(45, 2, 8, 256, d_v, prev, new, speca.ROUTE_AUTO, max_nodes=32)
     assert rel_err(cpu(d2.o), o_ref) <= TOL
-    assert rel_err(cpu(S), S_ref) <= TOL_FP32
+    assert rel_err(cpu(S), S_ref) <= TOL
+    d1.commit()
+    assert rel_err(cpu(S), cpu(d1.S)) <= 1e-4
+    for b in np.flatnonzero(p1.path_len == 0):
+        assert torch.equal(S[:, b], d1.S[:, b])
 
 
 def test_nothing_pending_and_nothing_to_verify():
