@@ -236,3 +236,18 @@ def test_fused_rounds_carry_the_state():
                  last.path_idx, last.path_len, last.status)
     S_ref = oracle.commit(S_ref, pl.k, pl.v, pl.alpha, pl.beta, pl.node_offsets, cpu(last.path_idx), cpu(last.path_len))
     assert rel_err(cpu(S), S_ref) <= TOL
+
+
+def test_more_sequences_than_the_walk_table_holds():
+    """Batches beyond the kernel's shared-memory walk table (128 sequences) take the global-memory
+    path for the per-sequence data: plain verification and the fused call on 150 sequences."""
+    rng = np.random.default_rng(17)
+    B = 150
+    prev = [synth.random_tree_parent(int(rng.integers(1, 13)), 4, 3, rng) for _ in range(B)]
+    new = [synth.random_tree_parent(int(rng.integers(1, 13)), 4, 3, rng) for _ in range(B)]
+    new[140] = np.zeros(0, np.int32)
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(47, 1, 2, 128, 128, prev, new, speca.ROUTE_FACTORIZED, max_nodes=16)
+    o1_ref = oracle.verify_tree(p1.S0, p1.q, p1.k, p1.v, p1.alpha, p1.beta, p1.node_offsets, p1.parent)
+    assert rel_err(cpu(d1.o), o1_ref) <= TOL
+    assert rel_err(cpu(d2.o), o_ref) <= TOL
+    assert rel_err(cpu(S), S_ref) <= TOL
