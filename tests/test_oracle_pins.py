@@ -287,6 +287,43 @@ def test_root_to_leaf_replay_equals_tree_verify():
         assert np.array_equal(oc[:, -1], o[:, t])
 
 
+def test_delayed_update_identities():
+    """What the fused commit-and-verify relies on (Section 5.2, Eq. 3):
+    (1) committing an accepted path and verifying a new draft from the committed state equals verifying
+        the tree obtained by hanging the new draft under the last accepted node, restricted to the new nodes;
+    (2) the committed state is gamma_A S0 + sum_i (gamma_A / gamma_i) u_i k_i^T, with u_i = beta_i (v_i - alpha_i S_{i-1} k_i)
+        the corrected values of the accepted nodes -- checked here with numpy only from the dense rule."""
+    rng = np.random.default_rng(31)
+    par1 = synth.random_tree_parent(11, 5, 3, rng)
+    par2 = synth.random_tree_parent(9, 4, 3, rng)
+    p1 = synth.make_problem(31, 2, 2, 16, 8, [par1])
+    p2 = synth.make_problem(32, 2, 2, 16, 8, [par2])
+    path = synth.root_path(par1, 10)
+    A = len(path)
+    idx = np.full((1, 8), -1, np.int32); idx[0, :A] = path
+    S1 = oracle.commit(p1.S0, p1.k, p1.v, p1.alpha, p1.beta, p1.node_offsets, idx, np.array([A], np.int32))
+    o_new = oracle.verify_tree(S1, p2.q, p2.k, p2.v, p2.alpha, p2.beta, p2.node_offsets, p2.parent)
+    # (1) spliced tree: accepted path as a chain, then the new nodes with their roots under its last node
+    sel = np.array(path)
+    cat = lambda a, b: np.concatenate([a[:, sel], b], axis=1)
+    par_sp = np.concatenate([np.arange(-1, A - 1), np.where(par2 < 0, A - 1, par2 + A)]).astype(np.int32)
+    o_sp = oracle.verify_tree(p1.S0, cat(p1.q, p2.q), cat(p1.k, p2.k), cat(p1.v, p2.v), cat(p1.alpha, p2.alpha),
+                              cat(p1.beta, p2.beta), np.array([0, A + len(par2)], np.int32), par_sp)
+    assert np.allclose(o_sp[:, A:], o_new, rtol=1e-12, atol=1e-14)
+    # (2) rank-A form of the committed state, unit (layer 1, head 0)
+    S0, q, k, v, al, be, _ = unit_arrays(p1, l=1, b=0, h=0)
+    S, us, gam = S0.copy(), [], []
+    g = 1.0
+    for t in path:
+        us.append(be[t] * (v[t] - al[t] * (S @ k[t])))
+        S = dense_rule(S, k[t], v[t], al[t], be[t])
+        g *= al[t]
+        gam.append(g)
+    S_rank = g * S0 + sum((g / gam[i]) * np.outer(us[i], k[t]) for i, t in enumerate(path))
+    assert np.allclose(S_rank, S, rtol=1e-12, atol=1e-14)
+    assert np.allclose(S1[1, 0, 0], S, rtol=1e-12, atol=1e-14)
+
+
 def test_sibling_isolation():
     """Changing any factor of node t changes outputs of t and its descendants only (tree mask, Section 4.2)."""
     rng = np.random.default_rng(13)
