@@ -79,6 +79,14 @@ constexpr int kUpdWarps = SPECA_UPD_WARPS;                   // state-update rol
 constexpr int kUpdThreads = kUpdWarps * 32;
 constexpr int kThreadsFused = kThreads + kUpdThreads;
 constexpr int kPrepThreads = 128;
+// The tensor core reads an fp32 state element as TF32 by dropping its low 13 mantissa bits, i.e. it
+// rounds every element toward zero: on average a value with mantissa m in [1, 2) loses 2^-11 / m of
+// itself, and E[1/m] is 0.69 .. 0.72 for any smooth distribution that spans a few binades.  The
+// products R = K S0^T and G = Q S0^T are therefore short by that fraction on average; the coefficients
+// that multiply them carry the expected-value correction.  It halves the typical error of the route
+// (measured 4.0e-4 -> 2.1e-4 at S0 ~ N(0, 0.02^2)); on a state whose elements happen to be exact in TF32
+// it costs at most the same 3.5e-4 of |R|, far inside the 2e-3 bar.
+constexpr float kDebias = 1.0f + 0.71f / 2048.0f;
 constexpr int kEpiChunk = 4;                   // nodes per TMEM read in the epilogue
 constexpr int kGramHalf = 32;                  // Gram columns parked per extraction pass
 constexpr int kStageChunkBytes = kBopRows * 128; // 64 bf16 columns of all [K;Q] rows: 16 KiB
@@ -967,7 +975,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     c[7] = active ? -sgn : 0.f;                                       // cV = beta
                     reinterpret_cast<float4 *>(cf)[0] = make_float4(c[0], c[1], c[2], c[3]);
                     reinterpret_cast<float4 *>(cf)[1] = make_float4(c[4], c[5], c[6], c[7]);
-                    cf[16] = active ? sgn * ratio : 0.f;                              // cR = -beta gamma
+                    cf[16] = active ? sgn * ratio * kDebias : 0.f;                              // cR = -beta gamma
                 } else {
                     // level d-1 is the node itself: (q_t . k_t) with ratio 1
                     c[7] = 0.f;
@@ -976,7 +984,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                         if (active && j == d - 1) c[j] = sgn * gsel[j];
                     reinterpret_cast<float4 *>(cf)[2] = make_float4(c[0], c[1], c[2], c[3]);
                     reinterpret_cast<float4 *>(cf)[3] = make_float4(c[4], c[5], c[6], c[7]);
-                    cf[17] = active ? sgn * ratio : 0.f;                              // cG = scale gamma
+                    cf[17] = active ? sgn * ratio * kDebias : 0.f;                              // cG = scale gamma
                     cf[18] = __int_as_float(active ? d - 1 : -1);
                     cf[19] = __int_as_float(active ? node * p.H * p.DV : 0);          // offset of the node's row
                 }
