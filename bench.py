@@ -322,6 +322,27 @@ def run_speca(args):
     dec_bytes = L * B * H * (2 * 4 * dk * dv + 4 * dk + 2 * dv + 8 + 4 * dv)
     del S_dec
 
+    # --- convolution-state commit (the other half of the state holder), same accepted paths --------
+    ch, W = H * (2 * dk + dv), 3
+    C = torch.zeros(L, B, W, ch, dtype=torch.bfloat16, device=dev)
+    p0 = pool[0]
+    x_conv = torch.zeros(L, p0["T"], ch, dtype=torch.bfloat16, device=dev)
+    speca.greedy_accept(B, 8, p0["d_offs"], p0["d_parent"], p0["d_draft"], p0["d_target"], p0["d_root"],
+                        path_idx, path_len, next_tok, status)
+    for _ in range(3):
+        speca.commit_conv(C, x_conv, p0["d_offs"], p0["T"], path_idx, path_len, status)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(10):
+        speca.commit_conv(C, x_conv, p0["d_offs"], p0["T"], path_idx, path_len, status)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    conv_ms = e0.elapsed_time(e1) / 10
+    pl0 = p0["path_len"]
+    conv_bytes = L * ch * 2 * int(np.sum(np.where(pl0 > 0, W + np.maximum(W - pl0, 0) + np.minimum(pl0, W), 0)))
+    del C, x_conv
+
     # --- the same rounds with the commit delayed into the next round's verification ----
     fused = None
     if not args.no_fused:
@@ -366,6 +387,8 @@ def run_speca(args):
                         "token_layers_per_s": B * L / (dec_ms * 1e-3),
                         "note": "one autoregressive token per sequence at the same batch"},
         "gpu_launches": 4 * K,
+        "conv_commit": {"ms": conv_ms, "channels": ch, "width": W, "gbs": conv_bytes / (conv_ms * 1e-3) / 1e9,
+                        "note": "speca_commit_conv on the accepted paths of one round; outside the timed step"},
         "fused": fused,
         "clocks": clocks,
         "e2e": e2e,

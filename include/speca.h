@@ -210,6 +210,22 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S,
                              void *workspace, size_t workspace_bytes,
                              int32_t *status_word, void *stream);
 
+/* Commit of the convolution state (Section 7: the state holder keeps (S, C); Section 8.4 checks that C
+ * is reproduced exactly).  The GDN layer is preceded by a causal depthwise convolution whose state is the
+ * last W = kernel_size - 1 inputs of every channel:
+ *      C   bf16 [L][B][W][channels]   oldest input first, updated in place
+ *      x   bf16 [L][T][channels]      inputs of the draft nodes (same packing as q, k, v)
+ * For every sequence the inputs of the accepted nodes path_idx[b][0..path_len[b]) are shifted into the
+ * register in path order: C becomes the last W rows of (old C rows, then the accepted rows).  16-bit
+ * patterns are copied, so the result is exact.  path_len[b] == 0 leaves the sequence's C untouched; a path
+ * with an index outside the sequence or longer than max_depth sets STATUS_BAD_PATH / TOO_DEEP and skips it.
+ * channels must be a multiple of 8, 1 <= W <= 8; C and x 16-byte aligned. */
+int speca_commit_conv(int32_t n_layers, int32_t batch, int32_t channels, int32_t width, int32_t max_depth,
+                      uint16_t *C, const uint16_t *x,
+                      const int32_t *node_offsets, int32_t total_nodes,
+                      const int32_t *path_idx, const int32_t *path_len,
+                      int32_t *status_word, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Variant of speca_verify_tree for callers that cannot provide scratch memory.
  * (The paper has no counterpart: this is a property of the library, not of the method.)

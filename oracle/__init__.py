@@ -147,3 +147,28 @@ def commit(S, k, v, alpha, beta, node_offsets, path_idx, path_len):
     if rc != 0:
         raise ValueError(f"oracle_commit: bad path (code {rc})")
     return S
+
+
+def commit_conv(C, x, node_offsets, path_idx, path_len):
+    """Convolution state of the causal depthwise convolution in front of the GDN layer (Section 7: the
+    state holder keeps (S, C)).  C [L,B,W,channels] are the last W = kernel_size - 1 inputs of every
+    channel, oldest first; x [L,T,channels] the inputs of the draft nodes.  Feeding the accepted nodes
+    through the convolution one by one shifts the register by one and appends the node's input; that
+    is done here literally, token by token.  16-bit patterns are moved, never interpreted.
+    Returns the new C (the input is not modified)."""
+    C = np.array(C, copy=True)
+    L, B, W, ch = C.shape
+    node_offsets = _c(node_offsets, np.int32)
+    path_idx, path_len = _c(path_idx, np.int32), _c(path_len, np.int32)
+    assert x.shape[0] == L and x.shape[2] == ch and x.dtype == C.dtype
+    for b in range(B):
+        base, n = int(node_offsets[b]), int(node_offsets[b + 1] - node_offsets[b])
+        for d in range(int(path_len[b])):
+            t = int(path_idx[b, d])
+            if not 0 <= t < n:
+                raise ValueError("commit_conv: bad path")
+            for l in range(L):
+                for w in range(W - 1):
+                    C[l, b, w] = C[l, b, w + 1]
+                C[l, b, W - 1] = x[l, base + t]
+    return C

@@ -25,7 +25,7 @@ ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
-           "speca_verify_tree_noalloc", "speca_commit_verify_tree"]
+           "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"]
 NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
@@ -82,8 +82,9 @@ def lib() -> ctypes.CDLL:
         L.speca_commit.argtypes = [dp] + [vp] * 6 + [i32] + [vp] * 5
         L.speca_commit_verify_tree.argtypes = ([dp] + [vp] * 7 + [i32] + [vp] * 3 + [vp] * 6 + [i32] + [vp] * 5 +
                                                [sz, vp, vp])
+        L.speca_commit_conv.argtypes = [i32] * 5 + [vp, vp, vp, i32, vp, vp, vp, vp]
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
-                     "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree"):
+                     "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -236,3 +237,17 @@ def commit_verify_tree(dims: Dims, S, prev, path_idx, path_len, q, k, v, alpha, 
         _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(),
         _ptr(status, i32, (1,), "status"), _stream())
     _check(rc, "speca_commit_verify_tree")
+
+
+def commit_conv(C, x, node_offsets, total_nodes, path_idx, path_len, status) -> None:
+    """speca_commit_conv: shift the inputs of the accepted nodes into the convolution state.
+    C bf16 [L,B,W,channels] (in place), x bf16 [L,T,channels]."""
+    L, B, W, ch = C.shape
+    T = int(total_nodes)
+    i32 = torch.int32
+    rc = lib().speca_commit_conv(
+        int(L), int(B), int(ch), int(W), int(path_idx.shape[1]), _ptr(C, torch.bfloat16, (L, B, W, ch), "C"),
+        _ptr(x, torch.bfloat16, (L, T, ch), "x"), _ptr(node_offsets, i32, (B + 1,), "node_offsets"), T,
+        _ptr(path_idx, i32, (B, path_idx.shape[1]), "path_idx"), _ptr(path_len, i32, (B,), "path_len"),
+        _ptr(status, i32, (1,), "status"), _stream())
+    _check(rc, "speca_commit_conv")

@@ -223,6 +223,20 @@ int speca_commit(const speca_dims *dims, float *S, const uint16_t *k, const uint
     return cuda_rc(launch_commit(p, dims->d_k, static_cast<cudaStream_t>(stream)));
 }
 
+int speca_commit_conv(int32_t n_layers, int32_t batch, int32_t channels, int32_t width, int32_t max_depth,
+                      uint16_t *C, const uint16_t *x, const int32_t *node_offsets, int32_t total_nodes,
+                      const int32_t *path_idx, const int32_t *path_len, int32_t *status_word, void *stream)
+{
+    if (!C || !x || !node_offsets || !path_idx || !path_len || !status_word) return SPECA_ERR_NULL;
+    if (n_layers < 1 || batch < 1 || total_nodes < 0 || max_depth < 1 || max_depth > 16) return SPECA_ERR_RANGE;
+    if (1LL * n_layers * batch > 0x7fffffffLL) return SPECA_ERR_RANGE;
+    if (channels < 8 || channels % 8 != 0 || width < 1 || width > 8) return SPECA_ERR_UNSUPPORTED;
+    if (misaligned(C) || misaligned(x)) return SPECA_ERR_ALIGN;
+    if (total_nodes == 0) return SPECA_OK;
+    return cuda_rc(launch_conv_commit(n_layers, batch, channels, width, total_nodes, max_depth, C, x, node_offsets,
+                                      path_idx, path_len, status_word, static_cast<cudaStream_t>(stream)));
+}
+
 int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k_prev, const uint16_t *v_prev,
                              const float *alpha_prev, const float *beta_prev, const float *u_prev_or_null,
                              const int32_t *node_offsets_prev, int32_t total_nodes_prev,

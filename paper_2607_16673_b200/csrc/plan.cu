@@ -227,7 +227,59 @@ pending_check_kernel(int32_t B, int32_t Tp, int32_t max_depth, int32_t max_len, 
     rec[9] = base;
 }
 
+// Convolution-state commit: one CTA per (layer, sequence), a thread per 8 channels.  A thread reads the
+// W rows that make up the new register (old rows and accepted inputs) into registers, then writes them,
+// so the in-place update never reads a row it has already overwritten.
+constexpr int kConvMaxWidth = 8;
+__global__ void __launch_bounds__(256)
+conv_commit_kernel(int32_t B, int32_t channels, int32_t W, int32_t T, int32_t max_depth, uint4 *__restrict__ C,
+                   const uint4 *__restrict__ x, const int32_t *__restrict__ node_offsets,
+                   const int32_t *__restrict__ path_idx, const int32_t *__restrict__ path_len, int32_t *status)
+{
+    const int l = blockIdx.x / B, b = blockIdx.x % B;
+    const int A = path_len[b];
+    if (A == 0) return;
+    const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+    int fault = 0;
+    if (A < 0 || A > max_depth) fault = SPECA_STATUS_TOO_DEEP;
+    else if (base < 0 || n < 0 || base + n > T) fault = SPECA_STATUS_BAD_OFFSETS;
+    else
+        for (int d = 0; d < A; ++d) {
+            const int t = path_idx[b * max_depth + d];
+            if (t < 0 || t >= n) fault = SPECA_STATUS_BAD_PATH;
+        }
+    if (fault) {
+        if (threadIdx.x == 0 && l == 0) atomicOr(status, fault);
+        return;
+    }
+    const int vec = channels / 8;                       // 16-byte pieces per row
+    uint4 *Cb = C + (size_t(l) * B + b) * W * vec;
+    for (int c = threadIdx.x; c < vec; c += blockDim.x) {
+        uint4 row[kConvMaxWidth];
+#pragma unroll
+        for (int w = 0; w < kConvMaxWidth; ++w) {
+            if (w < W) {
+                const int s = A + w;                    // index in (old rows, accepted rows); the last W are kept
+                if (s < W) row[w] = Cb[s * vec + c];
+                else row[w] = __ldg(x + (size_t(l) * T + base + path_idx[b * max_depth + (s - W)]) * vec + c);
+            }
+        }
+#pragma unroll
+        for (int w = 0; w < kConvMaxWidth; ++w)
+            if (w < W) Cb[w * vec + c] = row[w];
+    }
+}
+
 }  // namespace
+
+int launch_conv_commit(int32_t L, int32_t B, int32_t channels, int32_t W, int32_t T, int32_t max_depth, void *C,
+                       const void *x, const int32_t *node_offsets, const int32_t *path_idx, const int32_t *path_len,
+                       int32_t *status, cudaStream_t st)
+{
+    conv_commit_kernel<<<L * B, 256, 0, st>>>(B, channels, W, T, max_depth, static_cast<uint4 *>(C),
+                                              static_cast<const uint4 *>(x), node_offsets, path_idx, path_len, status);
+    return int(cudaGetLastError());
+}
 
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st)
 {

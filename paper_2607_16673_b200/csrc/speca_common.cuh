@@ -99,6 +99,9 @@ bool factorized_supported(const speca_dims *d);
 bool factorized_fused_supported(const speca_dims *d);
 int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st);
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
+int launch_conv_commit(int32_t L, int32_t B, int32_t channels, int32_t W, int32_t T, int32_t max_depth, void *C,
+                       const void *x, const int32_t *node_offsets, const int32_t *path_idx, const int32_t *path_len,
+                       int32_t *status, cudaStream_t st);
 int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
                   const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
                   int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,

@@ -459,6 +459,49 @@ def test_accept_batched_offsets():
 # ---------------------------------------------------------------------------
 # sizes the paper prints (pin the layouts and the record contents)
 # ---------------------------------------------------------------------------
+def test_conv_state_commit_hand_cases_and_convolution_identity():
+    """The convolution state is a shift register of the last W inputs (kernel size W + 1).  Hand cases,
+    and the property that defines it: the next token's causal convolution output computed from the
+    committed register equals the direct convolution (numpy.convolve) over the whole input history."""
+    u16 = lambda *v: np.array(v, np.uint16)
+    C = u16(1, 2, 3).reshape(1, 1, 3, 1)
+    x = u16(10, 11, 12, 13, 14).reshape(1, 5, 1)
+    offs = np.array([0, 5], np.int32)
+    idx = lambda *p: np.array([list(p) + [-1] * (8 - len(p))], np.int32)
+    run = lambda p: oracle.commit_conv(C, x, offs, idx(*p), np.array([len(p)], np.int32))[0, 0, :, 0].tolist()
+    assert run([]) == [1, 2, 3]
+    assert run([0]) == [2, 3, 10]
+    assert run([0, 2]) == [3, 10, 12]
+    assert run([0, 2, 3]) == [10, 12, 13]
+    assert run([0, 1, 2, 4]) == [11, 12, 14]
+    # convolution identity on random data: 2 layers, 3 sequences, kernel size 4, 5 channels
+    rng = np.random.default_rng(41)
+    L, B, W, ch = 2, 3, 3, 5
+    parents = [synth.random_tree_parent(9, 5, 3, rng), synth.chain_parent(2), synth.random_tree_parent(6, 6, 2, rng)]
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    T = int(offs[-1])
+    hist = rng.standard_normal((L, B, 7, ch)).astype(np.float32)                # inputs seen before the draft
+    Cb = synth.f32_to_bf16_bits(hist[:, :, -W:])
+    xb = synth.f32_to_bf16_bits(rng.standard_normal((L, T, ch)).astype(np.float32))
+    paths = [synth.root_path(parents[0], 8), [], synth.root_path(parents[2], 5)]
+    pidx = np.full((B, 8), -1, np.int32); plen = np.zeros(B, np.int32)
+    for b, pth in enumerate(paths):
+        pidx[b, :len(pth)] = pth; plen[b] = len(pth)
+    Cn = oracle.commit_conv(Cb, xb, offs, pidx, plen)
+    wts = rng.standard_normal((ch, W + 1))                                      # taps, newest input last
+    nxt = rng.standard_normal((L, B, ch))                                       # the next token's input
+    f = lambda bits: synth.bf16_bits_to_f32(bits).astype(np.float64)
+    for l in range(L):
+        for b in range(B):
+            seq = np.concatenate([f(synth.f32_to_bf16_bits(hist[l, b])), f(xb[l, offs[b] + np.array(paths[b], int)]).reshape(-1, ch),
+                                  nxt[l, b][None]], axis=0)
+            for c in range(ch):
+                direct = np.convolve(seq[:, c], wts[c, ::-1])[len(seq) - 1]         # causal output at the last position
+                from_state = np.dot(wts[c, :W], f(Cn[l, b, :, c])) + wts[c, W] * nxt[l, b, c]
+                assert abs(direct - from_state) <= 1e-12 * (1 + abs(direct))
+    assert np.array_equal(Cn[:, 1], Cb[:, 1])                                   # nothing accepted: untouched
+
+
 def test_paper_byte_counts():
     vals = {}
     for r in open(os.path.join(GOLDEN, "paper_sizes.txt")):
