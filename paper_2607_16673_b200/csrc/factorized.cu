@@ -1068,6 +1068,15 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     const int off = __float_as_int(coef[(p0 + i) * kCoefStride + 19]);   // p0 + i < npad; in floats of o
                     vv[i] = __ldg(v_row + off / TP);
                 }
+                // the value rows of the chunk after this one: into L1 now, so that their loads are short
+                // (a global load takes a microsecond or more while the state stream saturates HBM)
+                if (p0 + kEpiChunk < n) {
+#pragma unroll
+                    for (int i = 0; i < kEpiChunk; ++i) {
+                        const int offn = __float_as_int(coef[(p0 + kEpiChunk + i) * kCoefStride + 19]);
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(v_row + offn / TP));
+                    }
+                }
             };
             auto process = [&](int p0, const float (&R)[TP][kEpiChunk], const float (&G)[TP][kEpiChunk],
                                const VPack (&vv)[kEpiChunk]) {
