@@ -53,7 +53,7 @@ def parse_args():
                     help="cfg5 (default), cfg4, or 'paper': the paper's own target shape and proposal shapes (Table 1)")
     ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
     ap.add_argument("--route", type=int, default=0, help="0 auto, 1 serial, 2 factorized")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the fused commit-and-verify leg")
@@ -470,49 +470,76 @@ NCU_TRAFFIC = {"verify": 12 * 835.9e6, "commit": 12 * 716.9e6}     # 2-layer cap
 def run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream):
     """Same step, but every step's draft inputs start in pinned HOST memory and its results
     (outputs o, accepted paths, next tokens) are read back to the host inside the timed region.
-    The committed state is the durable device-resident object and stays in HBM."""
+    The committed state is the durable device-resident object and stays in HBM.  As a serving loop
+    would, the copies run on their own streams with two sets of device buffers, so that the upload
+    of step i+1, the kernels of step i and the read-back of step i-1 overlap (PCIe is full duplex)."""
     import torch
     L, B, H, dk, dv = dims.n_layers, dims.batch, dims.heads, dims.d_k, dims.d_v
     p0 = pool[0]
     T = p0["T"]
+    dev = S.device
     names = ["q", "k", "v", "alpha", "beta", "d_offs", "d_parent", "d_depth", "d_draft", "d_target", "d_root"]
     host = {n: torch.empty(p0[n].shape, dtype=p0[n].dtype, pin_memory=True).copy_(p0[n]) for n in names}
-    devb = {n: torch.empty_like(p0[n]) for n in names}
-    o = o_buf[: L * T * H * dv].view(L, T, H, dv)
-    o_host = torch.empty(o.shape, dtype=o.dtype, pin_memory=True)
+    devb = [{n: torch.empty_like(p0[n]) for n in names} for _ in range(2)]
+    o = [o_buf[: L * T * H * dv].view(L, T, H, dv), torch.empty(L, T, H, dv, dtype=torch.float32, device=dev)]
+    pi = [path_idx, torch.empty_like(path_idx)]
+    pl = [path_len, torch.empty_like(path_len)]
+    nt = [next_tok, torch.empty_like(next_tok)]
+    o_host = torch.empty(o[0].shape, dtype=torch.float32, pin_memory=True)
     pi_host = torch.empty(path_idx.shape, dtype=torch.int32, pin_memory=True)
     pl_host = torch.empty(path_len.shape, dtype=torch.int32, pin_memory=True)
     nt_host = torch.empty(next_tok.shape, dtype=torch.int32, pin_memory=True)
     h2d = sum(host[n].numel() * host[n].element_size() for n in names)
     d2h = sum(x.numel() * x.element_size() for x in (o_host, pi_host, pl_host, nt_host))
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_done = [torch.cuda.Event() for _ in range(2)]      # kernels of the step using buffer set j have finished
+    ev_out = [torch.cuda.Event() for _ in range(2)]       # results of buffer set j have reached the host
 
-    def one():
-        for n in names:
-            devb[n].copy_(host[n], non_blocking=True)
-        speca.verify_tree(dims, S, devb["q"], devb["k"], devb["v"], devb["alpha"], devb["beta"], devb["d_offs"], T,
-                          devb["d_parent"], devb["d_depth"], o, None, ws, status)
-        speca.greedy_accept(B, 8, devb["d_offs"], devb["d_parent"], devb["d_draft"], devb["d_target"], devb["d_root"],
-                            path_idx, path_len, next_tok, status)
-        speca.commit(dims, S, devb["k"], devb["v"], devb["alpha"], devb["beta"], devb["d_offs"], T, devb["d_parent"],
-                     path_idx, path_len, status)
-        o_host.copy_(o, non_blocking=True)
-        pi_host.copy_(path_idx, non_blocking=True)
-        pl_host.copy_(path_len, non_blocking=True)
-        nt_host.copy_(next_tok, non_blocking=True)
+    def one(i):
+        j = i & 1
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_done[j])                   # the step two back no longer reads these inputs
+            for n in names:
+                devb[j][n].copy_(host[n], non_blocking=True)
+            ev_in[j].record(s_in)
+        stream.wait_event(ev_in[j])
+        stream.wait_event(ev_out[j])                      # its results have been read back
+        d = devb[j]
+        speca.verify_tree(dims, S, d["q"], d["k"], d["v"], d["alpha"], d["beta"], d["d_offs"], T, d["d_parent"],
+                          d["d_depth"], o[j], None, ws, status)
+        speca.greedy_accept(B, 8, d["d_offs"], d["d_parent"], d["d_draft"], d["d_target"], d["d_root"], pi[j], pl[j],
+                            nt[j], status)
+        speca.commit(dims, S, d["k"], d["v"], d["alpha"], d["beta"], d["d_offs"], T, d["d_parent"], pi[j], pl[j], status)
+        ev_done[j].record(stream)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[j])
+            o_host.copy_(o[j], non_blocking=True)
+            pi_host.copy_(pi[j], non_blocking=True)
+            pl_host.copy_(pl[j], non_blocking=True)
+            nt_host.copy_(nt[j], non_blocking=True)
+            ev_out[j].record(s_out)
 
-    one()
+    for j in range(2):
+        ev_done[j].record(stream)
+        ev_out[j].record(stream)
+    one(0)
+    one(1)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n = max(1, args.e2e_steps)
+    n = max(2, args.e2e_steps)
     e0.record(stream)
-    for _ in range(n):
-        one()
+    for i in range(n):
+        one(i)
+    stream.wait_stream(s_out)
+    stream.wait_stream(s_in)
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / n
     return {"value": T * L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": n,
-            "note": "draft inputs from pinned host memory, outputs and accepted paths read back; state stays in HBM"}
+            "note": "draft inputs from pinned host memory, outputs and accepted paths read back, every step; uploads, "
+                    "kernels and read-backs of consecutive steps overlap on three streams; state stays in HBM"}
 
 
 # ---------------------------------------------------------------------------
