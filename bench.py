@@ -343,6 +343,37 @@ def run_speca(args):
     conv_bytes = L * ch * 2 * int(np.sum(np.where(pl0 > 0, W + np.maximum(W - pl0, 0) + np.minimum(pl0, W), 0)))
     del C, x_conv
 
+    # --- draft-side utilities on the same topology (context: they run once per round, before verification) ----
+    rng_u = np.random.default_rng(rank_seed(9000, rank))
+    logp = torch.from_numpy(np.log(rng_u.uniform(0.02, 1.0, p0["T"])).astype(np.float32)).to(dev)
+    mask_h = np.zeros((B, 64, 64), np.uint8)
+    for b_, par_ in enumerate(p0["parents"]):
+        for i_ in range(len(par_)):
+            a_ = i_
+            while a_ >= 0:
+                mask_h[b_, i_, a_] = 1
+                a_ = int(par_[a_])
+    mask_d = torch.from_numpy(mask_h).to(dev)
+    par_out = torch.empty(p0["T"], dtype=torch.int32, device=dev)
+    oo, op, oi = (torch.empty(B + 1, dtype=torch.int32, device=dev), torch.empty(p0["T"], dtype=torch.int32, device=dev),
+                  torch.empty(p0["T"], dtype=torch.int32, device=dev))
+
+    def time_util(fn, reps=10):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    mask_ms = time_util(lambda: speca.tree_mask_to_parent(mask_d, p0["d_offs"], par_out, status))
+    prune_ms = time_util(lambda: speca.prune_tree(64, 2.0, 32, p0["d_offs"], p0["d_parent"], logp, oo, op, oi, status))
+    assert torch.equal(par_out, p0["d_parent"]), "mask converter does not reproduce the parent array"
+
     # --- the same rounds with the commit delayed into the next round's verification ----
     fused = None
     if not args.no_fused:
@@ -389,6 +420,8 @@ def run_speca(args):
         "gpu_launches": 4 * K,
         "conv_commit": {"ms": conv_ms, "channels": ch, "width": W, "gbs": conv_bytes / (conv_ms * 1e-3) / 1e9,
                         "note": "speca_commit_conv on the accepted paths of one round; outside the timed step"},
+        "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms,
+                        "note": "one call over the batch's topology (tau = 2, budget 32); integer work outside the timed step"},
         "fused": fused,
         "clocks": clocks,
         "e2e": e2e,

@@ -210,6 +210,29 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S,
                              void *workspace, size_t workspace_bytes,
                              int32_t *status_word, void *stream);
 
+/* Draft-side utilities (integer work in front of the verification; Sections 6.1 and 7).
+ *
+ * speca_tree_mask_to_parent: the proposal converter.  mask uint8 [B][max_nodes][max_nodes]; for sequence b
+ * with n = node_offsets[b+1] - node_offsets[b] nodes, mask[b][i][j] != 0 (i, j < n) iff node j is node i
+ * or one of its ancestors (a drafter's tree attention mask).  Writes parent[node_offsets[b] + i] = the
+ * deepest strict ancestor of i (local index), -1 if it has none.  A mask that is not the mask of a tree in
+ * topological order sets STATUS_BAD_PARENT and leaves the sequence's parents untouched.
+ *
+ * speca_prune_tree: confidence-guided pruning.  logp float [T] are the drafter's step log-probabilities;
+ * q(v) is their sum over the root path of v (fp32, root first), q* its maximum over the sequence.  Kept are
+ * the nodes with q(v) >= q* - tau, of those the `budget` best by q (ties: lower index), and of those only
+ * nodes whose parent is kept -- with log-probabilities (<= 0) q never increases along a path and the last
+ * rule changes nothing.  The kept nodes of all sequences are written packed, in their original order:
+ * out_offsets [B+1], out_parent [.] (re-indexed, local), out_index [.] (original local index); out_parent
+ * and out_index need room for T entries.  A sequence with bad topology is reported and contributes nothing. */
+int speca_tree_mask_to_parent(int32_t batch, int32_t max_nodes, const uint8_t *mask,
+                              const int32_t *node_offsets, int32_t *parent,
+                              int32_t *status_word, void *stream);
+int speca_prune_tree(int32_t batch, int32_t max_nodes, float tau, int32_t budget,
+                     const int32_t *node_offsets, const int32_t *parent, const float *logp,
+                     int32_t *out_offsets, int32_t *out_parent, int32_t *out_index,
+                     int32_t *status_word, void *stream);
+
 /* Commit of the convolution state (Section 7: the state holder keeps (S, C); Section 8.4 checks that C
  * is reproduced exactly).  The GDN layer is preceded by a causal depthwise convolution whose state is the
  * last W = kernel_size - 1 inputs of every channel:

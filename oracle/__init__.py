@@ -172,3 +172,59 @@ def commit_conv(C, x, node_offsets, path_idx, path_len):
                     C[l, b, w] = C[l, b, w + 1]
                 C[l, b, W - 1] = x[l, base + t]
     return C
+
+
+def tree_mask_to_parent(mask, node_offsets):
+    """Proposal converter (Section 7): a drafter's tree attention mask -> parent array.  mask uint8
+    [B,N,N]; for sequence b with n nodes, mask[b,i,j] != 0 (i, j < n) iff node j is node i itself or one
+    of its ancestors.  The parent of i is its deepest strict ancestor, i.e. the one with the most
+    ancestors of its own; no strict ancestor -> -1.  Returns parent int32 [T] (local indices)."""
+    node_offsets = _c(node_offsets, np.int32)
+    B = node_offsets.shape[0] - 1
+    out = np.full(int(node_offsets[B]), -1, np.int32)
+    for b in range(B):
+        base, n = int(node_offsets[b]), int(node_offsets[b + 1] - node_offsets[b])
+        m = np.asarray(mask[b, :n, :n]) != 0
+        size = m.sum(axis=1)
+        for i in range(n):
+            best = -1
+            for j in range(n):
+                if j != i and m[i, j] and (best < 0 or size[j] > size[best]):
+                    best = j
+            out[base + i] = best
+    return out
+
+
+def prune_tree(node_offsets, parent, logp, tau, budget):
+    """Confidence-guided tree pruning (Section 6.1).  q(v) = sum of the step log-probabilities on the
+    root path of v (fp32, added root first); q* = max q; the window keeps q(v) >= q* - tau; of the
+    window the `budget` best by q are kept (ties: lower index first); a node whose parent was dropped is
+    dropped too, so the result is ancestor-closed whatever the scores.  Returns (out_offsets int32 [B+1],
+    out_parent int32 [T'], out_index int32 [T']): the kept nodes of every sequence in their original
+    order, parents re-indexed, and each kept node's original local index."""
+    node_offsets, parent = _c(node_offsets, np.int32), _c(parent, np.int32)
+    logp = _c(logp, np.float32)
+    B = node_offsets.shape[0] - 1
+    offs, out_parent, out_index = [0], [], []
+    for b in range(B):
+        base, n = int(node_offsets[b]), int(node_offsets[b + 1] - node_offsets[b])
+        par = parent[base:base + n]
+        q = np.zeros(n, np.float32)
+        for i in range(n):
+            q[i] = np.float32((q[par[i]] if par[i] >= 0 else np.float32(0)) + logp[base + i])
+        keep = np.zeros(n, bool)
+        if n:
+            thr = np.float32(q.max() - np.float32(tau))
+            window = [i for i in range(n) if q[i] >= thr]
+            window.sort(key=lambda i: (-float(q[i]), i))
+            keep[window[:max(int(budget), 0)]] = True
+            for i in range(n):
+                if par[i] >= 0 and not keep[par[i]]:
+                    keep[i] = False
+        new = np.cumsum(keep) - 1
+        for i in range(n):
+            if keep[i]:
+                out_parent.append(-1 if par[i] < 0 else int(new[par[i]]))
+                out_index.append(i)
+        offs.append(len(out_parent))
+    return np.asarray(offs, np.int32), np.asarray(out_parent, np.int32), np.asarray(out_index, np.int32)

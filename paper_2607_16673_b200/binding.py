@@ -25,7 +25,8 @@ ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
-           "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"]
+           "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv",
+           "speca_tree_mask_to_parent", "speca_prune_tree"]
 NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
@@ -83,6 +84,10 @@ def lib() -> ctypes.CDLL:
         L.speca_commit_verify_tree.argtypes = ([dp] + [vp] * 7 + [i32] + [vp] * 3 + [vp] * 6 + [i32] + [vp] * 5 +
                                                [sz, vp, vp])
         L.speca_commit_conv.argtypes = [i32] * 5 + [vp, vp, vp, i32, vp, vp, vp, vp]
+        L.speca_tree_mask_to_parent.argtypes = [i32, i32, vp, vp, vp, vp, vp]
+        L.speca_tree_mask_to_parent.restype = ctypes.c_int
+        L.speca_prune_tree.argtypes = [i32, i32, ctypes.c_float, i32] + [vp] * 8
+        L.speca_prune_tree.restype = ctypes.c_int
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
                      "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"):
             getattr(L, name).restype = ctypes.c_int
@@ -251,3 +256,29 @@ def commit_conv(C, x, node_offsets, total_nodes, path_idx, path_len, status) -> 
         _ptr(path_idx, i32, (B, path_idx.shape[1]), "path_idx"), _ptr(path_len, i32, (B,), "path_len"),
         _ptr(status, i32, (1,), "status"), _stream())
     _check(rc, "speca_commit_conv")
+
+
+def tree_mask_to_parent(mask, node_offsets, parent, status) -> None:
+    """speca_tree_mask_to_parent: mask uint8 [B,N,N] -> parent int32 [T] (written in place)."""
+    B, N, N2 = mask.shape
+    assert N == N2
+    rc = lib().speca_tree_mask_to_parent(int(B), int(N), _ptr(mask, torch.uint8, (B, N, N), "mask"),
+                                         _ptr(node_offsets, torch.int32, (B + 1,), "node_offsets"),
+                                         _ptr(parent, torch.int32, None, "parent"),
+                                         _ptr(status, torch.int32, (1,), "status"), _stream())
+    _check(rc, "speca_tree_mask_to_parent")
+
+
+def prune_tree(max_nodes: int, tau: float, budget: int, node_offsets, parent, logp, out_offsets, out_parent,
+               out_index, status) -> None:
+    """speca_prune_tree: keep the nodes within tau of the best cumulative log-probability, at most
+    `budget` per sequence; packed outputs."""
+    i32 = torch.int32
+    B = node_offsets.numel() - 1
+    T = parent.numel()
+    rc = lib().speca_prune_tree(int(B), int(max_nodes), float(tau), int(budget),
+                                _ptr(node_offsets, i32, (B + 1,), "node_offsets"), _ptr(parent, i32, (T,), "parent"),
+                                _ptr(logp, torch.float32, (T,), "logp"), _ptr(out_offsets, i32, (B + 1,), "out_offsets"),
+                                _ptr(out_parent, i32, (T,), "out_parent"), _ptr(out_index, i32, (T,), "out_index"),
+                                _ptr(status, i32, (1,), "status"), _stream())
+    _check(rc, "speca_prune_tree")

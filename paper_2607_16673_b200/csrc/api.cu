@@ -223,6 +223,26 @@ int speca_commit(const speca_dims *dims, float *S, const uint16_t *k, const uint
     return cuda_rc(launch_commit(p, dims->d_k, static_cast<cudaStream_t>(stream)));
 }
 
+int speca_tree_mask_to_parent(int32_t batch, int32_t max_nodes, const uint8_t *mask, const int32_t *node_offsets,
+                              int32_t *parent, int32_t *status_word, void *stream)
+{
+    if (!mask || !node_offsets || !parent || !status_word) return SPECA_ERR_NULL;
+    if (batch < 1 || max_nodes < 1 || max_nodes > 1024) return SPECA_ERR_RANGE;
+    return cuda_rc(launch_mask_to_parent(batch, max_nodes, mask, node_offsets, parent, status_word,
+                                         static_cast<cudaStream_t>(stream)));
+}
+
+int speca_prune_tree(int32_t batch, int32_t max_nodes, float tau, int32_t budget, const int32_t *node_offsets,
+                     const int32_t *parent, const float *logp, int32_t *out_offsets, int32_t *out_parent,
+                     int32_t *out_index, int32_t *status_word, void *stream)
+{
+    if (!node_offsets || !parent || !logp || !out_offsets || !out_parent || !out_index || !status_word)
+        return SPECA_ERR_NULL;
+    if (batch < 1 || max_nodes < 1 || max_nodes > 1024 || budget < 0 || !(tau >= 0.f)) return SPECA_ERR_RANGE;
+    return cuda_rc(launch_prune(batch, max_nodes, tau, budget, node_offsets, parent, logp, out_offsets, out_parent,
+                                out_index, status_word, static_cast<cudaStream_t>(stream)));
+}
+
 int speca_commit_conv(int32_t n_layers, int32_t batch, int32_t channels, int32_t width, int32_t max_depth,
                       uint16_t *C, const uint16_t *x, const int32_t *node_offsets, int32_t total_nodes,
                       const int32_t *path_idx, const int32_t *path_len, int32_t *status_word, void *stream)

@@ -270,7 +270,162 @@ conv_commit_kernel(int32_t B, int32_t channels, int32_t W, int32_t T, int32_t ma
     }
 }
 
+// Proposal converter: tree attention mask -> parent array.  One CTA per sequence, thread i owns node i:
+// its parent is the strict ancestor with the most ancestors of its own.  The mask is checked to be the mask
+// of a tree in topological order (self bit set, no later node among the ancestors, parent exactly one
+// level up); otherwise the sequence gets STATUS_BAD_PARENT and its parents are left untouched.
+__global__ void __launch_bounds__(256)
+mask_to_parent_kernel(int32_t N, const uint8_t *__restrict__ mask, const int32_t *__restrict__ node_offsets,
+                      int32_t *__restrict__ parent, int32_t *status)
+{
+    extern __shared__ int32_t sm[];                     // [N] ancestors-or-self per node, [N] parent
+    __shared__ int32_t s_flag;
+    const int b = blockIdx.x;
+    const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+    if (threadIdx.x == 0) s_flag = 0;
+    __syncthreads();
+    if (n < 0 || n > N) {
+        if (threadIdx.x == 0) atomicOr(status, n < 0 ? SPECA_STATUS_BAD_OFFSETS : SPECA_STATUS_TOO_MANY);
+        return;
+    }
+    const uint8_t *m = mask + size_t(b) * N * N;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        int cnt = 0, bad = m[size_t(i) * N + i] == 0;
+        for (int j = 0; j < n; ++j) {
+            const int on = m[size_t(i) * N + j] != 0;
+            cnt += on;
+            bad |= on && j > i;
+        }
+        sm[i] = cnt;
+        if (bad) atomicOr(&s_flag, 1);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        int best = -1;
+        for (int j = 0; j < n; ++j)
+            if (j != i && m[size_t(i) * N + j] != 0 && (best < 0 || sm[j] > sm[best])) best = j;
+        if (best >= 0 ? sm[best] != sm[i] - 1 : sm[i] != 1) atomicOr(&s_flag, 1);
+        sm[N + i] = best;
+    }
+    __syncthreads();
+    if (s_flag) {
+        if (threadIdx.x == 0) atomicOr(status, SPECA_STATUS_BAD_PARENT);
+        return;
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) parent[base + i] = sm[N + i];
+}
+
+// Confidence-guided pruning, step 1: one CTA per sequence selects its nodes and writes them, already
+// re-indexed, at the sequence's INPUT offset; out_offsets[b + 1] receives the count.  Scores are
+// accumulated in fp32 in node order, which adds every path root first, exactly as the definition does.
+__global__ void __launch_bounds__(128)
+prune_select_kernel(int32_t N, float tau, int32_t budget, const int32_t *__restrict__ node_offsets,
+                    const int32_t *__restrict__ parent, const float *__restrict__ logp, int32_t *__restrict__ out_offsets,
+                    int32_t *__restrict__ out_parent, int32_t *__restrict__ out_index, int32_t *status)
+{
+    extern __shared__ int32_t sm[];
+    float *q = reinterpret_cast<float *>(sm);           // [N]
+    int32_t *keep = sm + N, *newidx = sm + 2 * N;       // [N], [N]
+    __shared__ float s_thr;
+    __shared__ int32_t s_fault;
+    const int b = blockIdx.x;
+    const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+    if (threadIdx.x == 0) {
+        s_fault = 0;
+        if (n < 0 || base < 0) s_fault = SPECA_STATUS_BAD_OFFSETS;
+        else if (n > N) s_fault = SPECA_STATUS_TOO_MANY;
+        else {
+            float best = 0.f;
+            for (int i = 0; i < n; ++i) {
+                const int p = parent[base + i];
+                if (p < -1 || p >= i) { s_fault = SPECA_STATUS_BAD_PARENT; break; }
+                q[i] = (p >= 0 ? q[p] : 0.f) + logp[base + i];
+                best = (i == 0 || q[i] > best) ? q[i] : best;
+            }
+            s_thr = best - tau;
+        }
+    }
+    __syncthreads();
+    if (s_fault) {
+        if (threadIdx.x == 0) { atomicOr(status, s_fault); out_offsets[b + 1] = 0; }
+        return;
+    }
+    const float thr = s_thr;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const float qi = q[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const float qj = q[j];
+            rank += (qj >= thr) && (qj > qi || (qj == qi && j < i));
+        }
+        keep[i] = (qi >= thr) && rank < budget;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int c = 0;
+        for (int i = 0; i < n; ++i) {
+            const int p = parent[base + i];
+            if (p >= 0 && !keep[p]) keep[i] = 0;
+            newidx[i] = c;
+            c += keep[i];
+        }
+        out_offsets[b + 1] = c;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        if (keep[i]) {
+            const int p = parent[base + i];
+            out_parent[base + newidx[i]] = p < 0 ? -1 : newidx[p];
+            out_index[base + newidx[i]] = i;
+        }
+}
+
+// Step 2: one CTA turns the counts into offsets and closes the gaps, sequence by sequence in order
+// (a sequence only ever moves toward the front, over space earlier sequences have already left).
+__global__ void __launch_bounds__(256)
+prune_pack_kernel(int32_t B, const int32_t *__restrict__ node_offsets, int32_t *__restrict__ out_offsets,
+                  int32_t *__restrict__ out_parent, int32_t *__restrict__ out_index)
+{
+    __shared__ int32_t s_out;
+    if (threadIdx.x == 0) { s_out = 0; out_offsets[0] = 0; }
+    __syncthreads();
+    for (int b = 0; b < B; ++b) {
+        const int base = node_offsets[b], cnt = out_offsets[b + 1], dst = s_out;
+        __syncthreads();                                 // everyone has read the count before it becomes an offset
+        if (dst != base)
+            for (int i0 = 0; i0 < cnt; i0 += blockDim.x) {
+                const int i = i0 + threadIdx.x;
+                int vp = 0, vi = 0;
+                if (i < cnt) { vp = out_parent[base + i]; vi = out_index[base + i]; }
+                __syncthreads();                         // dst < base: a slice is read before it can be overwritten
+                if (i < cnt) { out_parent[dst + i] = vp; out_index[dst + i] = vi; }
+                __syncthreads();
+            }
+        if (threadIdx.x == 0) { s_out = dst + cnt; out_offsets[b + 1] = dst + cnt; }
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+int launch_mask_to_parent(int32_t B, int32_t N, const uint8_t *mask, const int32_t *node_offsets, int32_t *parent,
+                          int32_t *status, cudaStream_t st)
+{
+    mask_to_parent_kernel<<<B, 256, size_t(2 * N) * sizeof(int32_t), st>>>(N, mask, node_offsets, parent, status);
+    return int(cudaGetLastError());
+}
+
+int launch_prune(int32_t B, int32_t N, float tau, int32_t budget, const int32_t *node_offsets, const int32_t *parent,
+                 const float *logp, int32_t *out_offsets, int32_t *out_parent, int32_t *out_index, int32_t *status,
+                 cudaStream_t st)
+{
+    prune_select_kernel<<<B, 128, size_t(3 * N) * sizeof(int32_t), st>>>(N, tau, budget, node_offsets, parent, logp,
+                                                                        out_offsets, out_parent, out_index, status);
+    int e = int(cudaGetLastError());
+    if (e != 0) return e;
+    prune_pack_kernel<<<1, 256, 0, st>>>(B, node_offsets, out_offsets, out_parent, out_index);
+    return int(cudaGetLastError());
+}
 
 int launch_conv_commit(int32_t L, int32_t B, int32_t channels, int32_t W, int32_t T, int32_t max_depth, void *C,
                        const void *x, const int32_t *node_offsets, const int32_t *path_idx, const int32_t *path_len,

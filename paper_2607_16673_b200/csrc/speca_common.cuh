@@ -99,6 +99,11 @@ bool factorized_supported(const speca_dims *d);
 bool factorized_fused_supported(const speca_dims *d);
 int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st);
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
+int launch_mask_to_parent(int32_t B, int32_t N, const uint8_t *mask, const int32_t *node_offsets, int32_t *parent,
+                          int32_t *status, cudaStream_t st);
+int launch_prune(int32_t B, int32_t N, float tau, int32_t budget, const int32_t *node_offsets, const int32_t *parent,
+                 const float *logp, int32_t *out_offsets, int32_t *out_parent, int32_t *out_index, int32_t *status,
+                 cudaStream_t st);
 int launch_conv_commit(int32_t L, int32_t B, int32_t channels, int32_t W, int32_t T, int32_t max_depth, void *C,
                        const void *x, const int32_t *node_offsets, const int32_t *path_idx, const int32_t *path_len,
                        int32_t *status, cudaStream_t st);

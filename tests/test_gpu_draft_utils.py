@@ -1,0 +1,80 @@
+"""GPU parity of the draft-side integer utilities (tree-mask converter, confidence-guided pruning): bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_16673_b200 import binding as speca
+from paper_2607_16673_b200 import synth
+
+pytestmark = pytest.mark.gpu
+t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def mask_of(parents, N):
+    m = np.zeros((len(parents), N, N), np.uint8)
+    for b, par in enumerate(parents):
+        for i in range(len(par)):
+            for a in synth.root_path(par, i):
+                m[b, i, a] = 1
+    return m
+
+
+def batch(rng, B, lo, hi):
+    parents = [synth.random_tree_parent(int(rng.integers(lo, hi + 1)), 8, 4, rng) for _ in range(B)]
+    parents[B // 2] = np.zeros(0, np.int32)
+    parents[0] = np.array([-1, -1, 0, -1, 1], np.int32)
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    return parents, offs
+
+
+def test_tree_mask_to_parent():
+    rng = np.random.default_rng(61)
+    parents, offs = batch(rng, 40, 1, 64)
+    mask = mask_of(parents, 64)
+    T = int(offs[-1])
+    par = torch.full((T,), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    speca.tree_mask_to_parent(t(mask), t(offs), par, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(par.cpu().numpy(), oracle.tree_mask_to_parent(mask, offs))
+    assert np.array_equal(par.cpu().numpy(), np.concatenate(parents))
+    # a mask that is not a tree mask (node 3 of sequence 1 sees node 1 but not node 1's parent)
+    bad = mask.copy()
+    p1 = parents[1]
+    deep = int(np.argmax(synth.depth_of(p1)))
+    if synth.depth_of(p1)[deep] >= 3:
+        bad[1, deep, synth.root_path(p1, deep)[0]] = 0
+        par.fill_(-7)
+        speca.tree_mask_to_parent(t(bad), t(offs), par, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == speca.STATUS_BAD_PARENT
+        got = par.cpu().numpy()
+        assert np.all(got[offs[1]:offs[2]] == -7)
+        keep = np.r_[0:offs[1], offs[2]:T]
+        assert np.array_equal(got[keep], np.concatenate(parents)[keep])
+
+
+@pytest.mark.parametrize("tau,budget", [(0.5, 64), (1.25, 6), (3.0, 16), (10.0, 3), (0.0, 1), (2.0, 0)])
+def test_prune_tree(tau, budget):
+    rng = np.random.default_rng(62)
+    parents, offs = batch(rng, 50, 1, 64)
+    parent = np.concatenate(parents).astype(np.int32)
+    T = int(offs[-1])
+    # realistic scores: log-softmax-like values in fp32 (ties are rare), plus a block of exact ties
+    logp = np.log(rng.uniform(0.02, 1.0, T)).astype(np.float32)
+    logp[offs[3]:offs[4]] = -0.5
+    oo = torch.zeros(len(parents) + 1, dtype=torch.int32, device="cuda")
+    op = torch.full((T,), -7, dtype=torch.int32, device="cuda")
+    oi = torch.full((T,), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    speca.prune_tree(64, tau, budget, t(offs), t(parent), t(logp), oo, op, oi, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ro, rp, ri = oracle.prune_tree(offs, parent, logp, tau, budget)
+    assert np.array_equal(oo.cpu().numpy(), ro)
+    n = int(ro[-1])
+    assert np.array_equal(op.cpu().numpy()[:n], rp) and np.array_equal(oi.cpu().numpy()[:n], ri)
+    # the pruned topology is a valid input of the verification path
+    assert np.all(rp < np.arange(n) - ro[np.searchsorted(ro, np.arange(n), side="right") - 1]) or n == 0

@@ -502,6 +502,61 @@ def test_conv_state_commit_hand_cases_and_convolution_identity():
     assert np.array_equal(Cn[:, 1], Cb[:, 1])                                   # nothing accepted: untouched
 
 
+def _mask_of(parents, N):
+    """Tree attention mask built by walking every root path (independent of the converter)."""
+    m = np.zeros((len(parents), N, N), np.uint8)
+    for b, par in enumerate(parents):
+        for i in range(len(par)):
+            for a in synth.root_path(par, i):
+                m[b, i, a] = 1
+    return m
+
+
+def test_tree_mask_converter_round_trip():
+    rng = np.random.default_rng(51)
+    parents = [synth.random_tree_parent(int(rng.integers(1, 30)), 8, 4, rng) for _ in range(6)]
+    parents += [np.array([-1, -1, 0, -1, 1], np.int32), np.zeros(0, np.int32), synth.chain_parent(7)]
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    got = oracle.tree_mask_to_parent(_mask_of(parents, 32), offs)
+    assert np.array_equal(got, np.concatenate(parents))
+
+
+def test_pruning_hand_case_and_selection_properties():
+    """Section 6.1: window q >= q* - tau on cumulative log-probabilities, then the budget."""
+    #        0(-0.5)            3(-2.0)
+    #       /      \
+    #   1(-0.25)  2(-1.0)            q: 0:-0.5  1:-0.75  2:-1.5  3:-2.0  4:-0.875 (child of 1, -0.125)
+    par = np.array([-1, 0, 0, -1, 1], np.int32)
+    lp = np.array([-0.5, -0.25, -1.0, -2.0, -0.125], np.float32)
+    offs = np.array([0, 5], np.int32)
+    keep = lambda tau, T: oracle.prune_tree(offs, par, lp, tau, T)
+    o, p, idx = keep(0.4, 8)                          # window: q >= -0.9 -> nodes 0, 1, 4
+    assert idx.tolist() == [0, 1, 4] and p.tolist() == [-1, 0, 1] and o.tolist() == [0, 3]
+    assert keep(1.0, 8)[2].tolist() == [0, 1, 2, 4]   # q >= -1.5
+    assert keep(5.0, 8)[2].tolist() == [0, 1, 2, 3, 4]
+    assert keep(5.0, 2)[2].tolist() == [0, 1]         # budget cuts the score-ranked selection
+    assert keep(0.0, 8)[2].tolist() == [0]            # only q*
+    assert keep(5.0, 0)[2].tolist() == []
+    # properties on random trees with scores that are exact in fp32 (multiples of 1/8): the kept set is the
+    # top-`budget` of the window by (q, index) computed independently in float64 with Python's sort
+    rng = np.random.default_rng(52)
+    parents = [synth.random_tree_parent(int(rng.integers(1, 40)), 8, 4, rng) for _ in range(8)]
+    offs = np.concatenate([[0], np.cumsum([len(pp) for pp in parents])]).astype(np.int32)
+    parent = np.concatenate(parents)
+    logp = (-rng.integers(0, 12, int(offs[-1])) / 8.0).astype(np.float32)
+    for tau, T in [(0.5, 64), (1.25, 6), (3.0, 16), (10.0, 3)]:
+        oo, pp, ii = oracle.prune_tree(offs, parent, logp, tau, T)
+        for b, par in enumerate(parents):
+            n = len(par)
+            q = np.array([sum(float(logp[offs[b] + a]) for a in synth.root_path(par, i)) for i in range(n)])
+            window = sorted([i for i in range(n) if q[i] >= q.max() - tau], key=lambda i: (-q[i], i))[:T]
+            got = ii[oo[b]:oo[b + 1]].tolist()
+            assert got == sorted(window)
+            newpar = pp[oo[b]:oo[b + 1]]
+            for r, i in enumerate(got):                # ancestor-closed and re-indexed consistently
+                assert (par[i] < 0 and newpar[r] == -1) or got[newpar[r]] == par[i]
+
+
 def test_paper_byte_counts():
     vals = {}
     for r in open(os.path.join(GOLDEN, "paper_sizes.txt")):
