@@ -715,8 +715,34 @@ def run_paper_shapes(args):
         pidx[0, :len(path)] = t(np.asarray(path, np.int32))
         plen = torch.tensor([len(path)], dtype=torch.int32, device=dev)
         ms_commit = timed(lambda i: speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent, pidx, plen, status))
+        # the whole round (verify -> accept -> commit), launched kernel by kernel and replayed as ONE CUDA graph:
+        # at this size the round is launch-bound, and the entry points are capturable (no allocation, no
+        # synchronisation, all arguments fixed at capture)
+        draft, target, root = t(prob.draft_tok), t(prob.target_tok), t(prob.root_target_tok)
+        gp = torch.full((1, md), -1, dtype=torch.int32, device=dev)
+        gl = torch.zeros(1, dtype=torch.int32, device=dev)
+        gn = torch.zeros(1, dtype=torch.int32, device=dev)
+
+        def round_(i):
+            speca.verify_tree(dims, S[i % COPIES], q, k, v, al, be, offs, n, parent, None, o, None, ws, status)
+            speca.greedy_accept(1, md, offs, parent, draft, target, root, gp, gl, gn, status)
+            speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent, gp, gl, status)
+
+        ms_round = timed(round_)
+        graphs = []
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for c in range(COPIES):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    round_(c)
+                graphs.append(g)
+        stream.wait_stream(side)
+        ms_graph = timed(lambda i: graphs[i % COPIES].replay())
         assert int(status.item()) == 0
         rows.append({"top_k": top_k, "config_depth": depth, "nodes": n, "tree_depth": tree_depth,
+                     "round_ms": ms_round, "round_cuda_graph_ms": ms_graph,
                      "leaves": Br, "replayed_tokens": Tr, "verify_tree_ms": ms_tree, "r2l_replay_ms": ms_r2l,
                      "tree_vs_r2l": ms_r2l / ms_tree, "commit_ms": ms_commit, "accepted_len": len(path),
                      "token_layers_per_s": n * L / ((ms_tree + ms_commit) * 1e-3)})

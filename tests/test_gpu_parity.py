@@ -423,3 +423,30 @@ def test_factorized_key_width_256_batched_paper_shape():
     parents = [synth.proposal_tree_parent(4, int(rng.integers(3, 9)), int(rng.integers(8, 33)), rng) for _ in range(24)]
     prob = synth.make_problem(981, 2, 8, 256, 256, parents, name="paper-shape-batch")
     check_verify(prob, speca.ROUTE_AUTO, max_nodes=32)
+
+
+def test_round_is_cuda_graph_capturable():
+    """No entry point allocates or synchronises, so a whole round can be captured once and replayed."""
+    rng = np.random.default_rng(990)
+    prob = synth.make_problem(991, 2, 4, 128, 256, synth.ragged_tree_batch(rng, 4, 4, 40, 8))
+    eager = DevProblem(prob, route=speca.ROUTE_AUTO, max_nodes=64)
+    eager.verify_tree(); eager.accept(); eager.commit()
+    assert eager.status_value() == 0
+    dp = DevProblem(prob, route=speca.ROUTE_AUTO, max_nodes=64)
+    S0 = dp.S.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        dp.verify_tree(); dp.accept(); dp.commit()                 # warm-up outside the capture (first-call attributes)
+        dp.S.copy_(S0)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            dp.verify_tree(); dp.accept(); dp.commit()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        dp.S.copy_(S0)
+        dp.o.fill_(float("nan"))
+        g.replay()
+        assert dp.status_value() == 0
+        assert torch.equal(dp.o, eager.o) and torch.equal(dp.S, eager.S)
+        assert torch.equal(dp.path_idx, eager.path_idx) and torch.equal(dp.path_len, eager.path_len)
