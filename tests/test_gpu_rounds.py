@@ -110,3 +110,84 @@ def test_cfg5_full_size_sampled():
 
 def test_cfg4_full_size_sampled():
     run_rounds("cfg4", 24, 32, 2, speca.ROUTE_AUTO, TOL, n_sample=32, seed=92)
+
+
+def run_rounds_fused(kind, L, B, rounds, tol, n_sample=24, seed=177, H=16, dk=128, dv=256, max_nodes=64):
+    """The same loop through speca_commit_verify_tree: the commit of round r - 1 runs inside the
+    verification of round r; the last pending commit is flushed with speca_commit."""
+    dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, max_nodes, speca.ROUTE_AUTO)
+    S = synth.device_state(seed, L, B, H, dk, dv)
+    rng = np.random.default_rng(seed)
+    units = sorted({(int(rng.integers(L)), int(rng.integers(B // 2) + (B // 2) * (i % 2)), int(rng.integers(H)))
+                    for i in range(n_sample)})
+    S_ref = np.stack([S[l, b, h].cpu().numpy().astype(np.float64) for (l, b, h) in units])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    paths = [(torch.zeros(B, 8, dtype=torch.int32, device="cuda"), torch.zeros(B, dtype=torch.int32, device="cuda"))
+             for _ in range(2)]
+    next_tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    t = lambda a: torch.from_numpy(a).cuda()
+    worst_o = worst_s = 0.0
+    prev = prev_host = None
+    for r in range(rounds + 1):
+        flush = r == rounds
+        if not flush:
+            if kind == "paper256":
+                trng = np.random.default_rng(seed + 100 + r)
+                parents = [synth.chain_parent(8) for _ in range(B // 2)]
+                parents += [synth.proposal_tree_parent(4, int(trng.integers(4, 9)), int(trng.integers(16, 33)), trng, 8)
+                            for _ in range(B - B // 2)]
+                offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+                parent = np.concatenate(parents).astype(np.int32)
+                draft, target, root = synth.draw_tokens(trng, offs, parent, 0.75)
+            else:
+                parents, offs, parent, _, draft, target, root = host_topology(kind, B, seed + 100 + r)
+            T = int(offs[-1])
+            q, k, v, al, be = synth.device_records(seed + 200 + r, L, T, H, dk, dv)
+            d_offs, d_par = t(offs), t(parent)
+            o = torch.full((L, T, H, dv), float("nan"), device="cuda")
+            u = torch.empty(L, T, H, dv, device="cuda")
+            ws = speca.alloc_workspace(dims, T)
+        pi_d, pl_d = paths[r & 1]
+        ppi, ppl = paths[(r - 1) & 1]
+        # the oracle commits the previous round's paths to its own state first
+        if prev_host is not None:
+            sp0, sub_pi, sub_pl = prev_host
+            S_ref = oracle.commit(S_ref[None, :, None], sp0["k"], sp0["v"], sp0["alpha"], sp0["beta"], sp0["offs"],
+                                  sub_pi, sub_pl)[0, :, 0]
+        if flush:
+            pp = prev
+            speca.commit(dims, S, pp["k"], pp["v"], pp["alpha"], pp["beta"], pp["node_offsets"], pp["total_nodes"],
+                         pp["parent"], ppi, ppl, status)
+        else:
+            speca.commit_verify_tree(dims, S, prev, ppi, ppl, q, k, v, al, be, d_offs, T, d_par, None, o, u, ws, status)
+            speca.greedy_accept(B, 8, d_offs, d_par, t(draft), t(target), t(root), pi_d, pl_d, next_tok, status)
+        assert int(status.item()) == 0
+        S_gpu = np.stack([S[l, b, h].cpu().numpy() for (l, b, h) in units])
+        worst_s = max(worst_s, rel_err(S_gpu, S_ref))
+        if flush:
+            break
+        sp = sample_problem(units, parents, offs, S_ref, q, k, v, al, be, dk, dv)
+        o_ref = oracle.verify_tree(sp["S"], sp["q"], sp["k"], sp["v"], sp["alpha"], sp["beta"], sp["offs"], sp["parent"])
+        pi, pl, _ = oracle.greedy_accept(offs, parent, draft, target, root, 8)
+        assert np.array_equal(pi_d.cpu().numpy(), pi) and np.array_equal(pl_d.cpu().numpy(), pl)
+        o_gpu = np.concatenate([o[l, int(offs[b]):int(offs[b + 1]), h].cpu().numpy() for (l, b, h) in units])
+        assert not np.isnan(o_gpu).any()
+        worst_o = max(worst_o, rel_err(o_gpu, o_ref[0, :, 0]))
+        prev = dict(k=k, v=v, alpha=al, beta=be, u=u, node_offsets=d_offs, total_nodes=T, parent=d_par)
+        prev_host = (sp, np.stack([pi[b] for (_, b, _) in units]), np.asarray([pl[b] for (_, b, _) in units], np.int32))
+    print(f"fused {kind} L={L} B={B} rounds={rounds}: worst verify err {worst_o:.3e}, worst state err {worst_s:.3e}")
+    assert worst_o <= tol and worst_s <= tol
+    return worst_o, worst_s
+
+
+def test_fused_cfg5_shaped_16_rounds():
+    run_rounds_fused("cfg5", 2, 128, 16, TOL)
+
+
+def test_fused_paper256_shaped_rounds():
+    run_rounds_fused("paper256", 2, 64, 8, TOL, H=8, dk=256, dv=256, max_nodes=32)
+
+
+def test_fused_cfg5_full_size_sampled():
+    """The fused rounds in the benchmark's own launch configuration (6.4 GB of state), three rounds."""
+    run_rounds_fused("cfg5", 24, 128, 3, TOL, n_sample=32, seed=191)
