@@ -497,7 +497,7 @@ def run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, di
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant
 # kernels from the ncu captures summarised under profiles/; None until captured.
-NCU_TRAFFIC = {"verify": 12 * 835.9e6, "commit": 12 * 716.9e6}     # 2-layer captures x 12 (traffic is proportional to units)
+NCU_TRAFFIC = {"verify": 12 * 835.1e6, "commit": 12 * 716.9e6}     # 2-layer captures x 12 (traffic is proportional to units)
 
 
 def run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream):
