@@ -450,3 +450,29 @@ def test_round_is_cuda_graph_capturable():
         assert dp.status_value() == 0
         assert torch.equal(dp.o, eager.o) and torch.equal(dp.S, eager.S)
         assert torch.equal(dp.path_idx, eager.path_idx) and torch.equal(dp.path_len, eager.path_len)
+
+
+@pytest.mark.parametrize("route", ROUTES)
+def test_deltanet_records_are_the_alpha_one_case(route):
+    """A DeltaNet layer keeps (k, v, beta) and has no decay: the same entry points with alpha = 1
+    (Section 5.1, remark on other layer types).  Verify, commit and the fused call against the oracle."""
+    rng = np.random.default_rng(995)
+    p1 = synth.make_problem(996, 2, 4, 128, 128, synth.ragged_tree_batch(rng, 4, 4, 30, 8))
+    p2 = synth.make_problem(997, 2, 4, 128, 128, synth.ragged_tree_batch(rng, 4, 4, 30, 8))
+    p1.alpha[:] = 1.0
+    p2.alpha[:] = 1.0
+    d1, _ = check_verify(p1, route, want_u=True, max_nodes=64)
+    d1.accept()
+    pi, pl, _ = oracle.greedy_accept(p1.node_offsets, p1.parent, p1.draft_tok, p1.target_tok, p1.root_target_tok, 8)
+    d2 = DevProblem(p2, route=route, want_u=True, max_nodes=64)
+    S = d1.S.clone()
+    prev = dict(k=d1.k, v=d1.v, alpha=d1.alpha, beta=d1.beta, u=d1.u, node_offsets=d1.node_offsets, total_nodes=d1.T,
+                parent=d1.parent)
+    speca.commit_verify_tree(d2.dims, S, prev, d1.path_idx, d1.path_len, d2.q, d2.k, d2.v, d2.alpha, d2.beta,
+                             d2.node_offsets, d2.T, d2.parent, None, d2.o, d2.u, d2.ws, d2.status)
+    assert d2.status_value() == 0
+    S_ref = oracle_commit(p1, pi, pl)
+    o_ref = oracle.verify_tree(S_ref, p2.q, p2.k, p2.v, p2.alpha, p2.beta, p2.node_offsets, p2.parent)
+    assert rel_err(cpu(S), S_ref) <= tol_for(route) and rel_err(cpu(d2.o), o_ref) <= tol_for(route)
+    d1.commit()
+    assert rel_err(cpu(d1.S), S_ref) <= TOL_FP32
