@@ -87,6 +87,11 @@ extern "C" {
 #define SPECA_ROUTE_SERIAL      1   /* state-resident walk, one rank-1 update per node (Section 4.1) */
 #define SPECA_ROUTE_FACTORIZED  2   /* tree-masked WY form on tensor cores (Section 4.2)           */
 
+/* recurrences (dims.rule; Section 5.1, remark on other layer types).  A DeltaNet layer (k, v, beta, no
+ * decay) is the gated delta rule with alpha = 1 and needs no value of its own. */
+#define SPECA_RULE_GATED_DELTA     0   /* S' = S alpha (I - beta k k^T) + beta v k^T   (GDN)                   */
+#define SPECA_RULE_GATED_NO_ERASE  1   /* S' = alpha S + beta v k^T   (GLA-style: key, value, gate; no read-out) */
+
 typedef struct speca_dims {
     int32_t n_layers;    /* L >= 1                                                     */
     int32_t batch;       /* B >= 1                                                     */
@@ -97,6 +102,7 @@ typedef struct speca_dims {
     int32_t max_depth;   /* longest root path in nodes, 1..16; width of path_idx rows  */
     int32_t max_nodes;   /* node budget per sequence (Section 6.1), 1..1024            */
     int32_t route;       /* SPECA_ROUTE_*                                              */
+    int32_t rule;        /* SPECA_RULE_*: which recurrence the layer applies           */
 } speca_dims;
 
 int         speca_version(void);

@@ -47,6 +47,8 @@ def _load():
         lib = ctypes.CDLL(_LIB_PATH)
         i32, f64, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
         lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_set_rule.argtypes = [i32]
+        lib.oracle_set_rule.restype = None
         lib.oracle_decode_step.argtypes = [i32] * 5 + [f64] + [vp] * 7
         lib.oracle_verify_tree.argtypes = [i32] * 5 + [f64] + [vp] * 9
         lib.oracle_greedy_accept.argtypes = [i32, i32] + [vp] * 8
@@ -61,6 +63,15 @@ def _p(a: np.ndarray):
 
 def _c(a, dtype):
     return np.ascontiguousarray(a, dtype=dtype)
+
+
+RULE_GATED_DELTA, RULE_GATED_NO_ERASE = 0, 1
+
+
+def set_rule(rule: int) -> None:
+    """Select the recurrence for the following calls: RULE_GATED_DELTA (default; DeltaNet is its alpha = 1
+    case) or RULE_GATED_NO_ERASE, S' = alpha S + beta v k^T (GLA-style layers; Section 5.1, remark)."""
+    _load().oracle_set_rule(int(rule))
 
 
 def num_threads() -> int:

@@ -51,9 +51,17 @@ static double bf16_to_double(uint16_t h)
     return (double)f;
 }
 
-/* One application of the gated delta rule to one head's state, in place.
+/* Which recurrence the entry points apply (Section 5.1, remark on other layer types):
+ *   0  gated delta rule (GDN; a DeltaNet layer is its alpha = 1 case)
+ *   1  gated rule without the erase term,  S' = alpha S + beta v k^T  (GLA-style layers, which keep
+ *      key, value and gate but no delta-rule read-out)
+ * Set between calls with oracle_set_rule; read-only while a call runs. */
+static int g_rule = 0;
+void oracle_set_rule(int rule) { g_rule = rule; }
+
+/* One application of the rule to one head's state, in place.
  * Order of the definition: decay the state, read it with the key, erase that
- * read-out, write the new value.  S is [d_v][d_k]. */
+ * read-out (rule 0 only), write the new value.  S is [d_v][d_k]. */
 static void gdn_rule(int d_k, int d_v, double *S, const double *k, const double *v,
                      double alpha, double beta)
 {
@@ -61,7 +69,8 @@ static void gdn_rule(int d_k, int d_v, double *S, const double *k, const double 
         double *row = S + (size_t)i * d_k;
         for (int j = 0; j < d_k; ++j) row[j] *= alpha;          /* S alpha            */
         double read = 0.0;
-        for (int j = 0; j < d_k; ++j) read += row[j] * k[j];    /* (S alpha) k        */
+        if (g_rule == 0)
+            for (int j = 0; j < d_k; ++j) read += row[j] * k[j];    /* (S alpha) k        */
         for (int j = 0; j < d_k; ++j)                            /* - beta (.) k^T + beta v k^T */
             row[j] += beta * (v[i] - read) * k[j];
     }

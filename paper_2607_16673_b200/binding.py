@@ -22,6 +22,7 @@ OK = 0
 STATUS_BAD_PARENT, STATUS_BAD_OFFSETS, STATUS_BAD_PATH, STATUS_TOO_DEEP = 1, 2, 4, 8
 STATUS_TOO_MANY, STATUS_TIMEOUT, STATUS_BAD_DEPTH = 16, 32, 64
 ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
+RULE_GATED_DELTA, RULE_GATED_NO_ERASE = 0, 1
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
@@ -37,7 +38,8 @@ class SpecaError(RuntimeError):
 class _Dims(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("heads", ctypes.c_int32),
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("scale", ctypes.c_float),
-                ("max_depth", ctypes.c_int32), ("max_nodes", ctypes.c_int32), ("route", ctypes.c_int32)]
+                ("max_depth", ctypes.c_int32), ("max_nodes", ctypes.c_int32), ("route", ctypes.c_int32),
+                ("rule", ctypes.c_int32)]
 
 
 @dataclass
@@ -51,10 +53,11 @@ class Dims:
     max_depth: int = 8
     max_nodes: int = 64
     route: int = ROUTE_AUTO
+    rule: int = 0
 
     def c(self) -> _Dims:
         return _Dims(self.n_layers, self.batch, self.heads, self.d_k, self.d_v, self.scale,
-                     self.max_depth, self.max_nodes, self.route)
+                     self.max_depth, self.max_nodes, self.route, self.rule)
 
 
 _lib = None

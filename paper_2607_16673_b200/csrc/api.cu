@@ -16,6 +16,7 @@ int check_dims(const speca_dims *d)
     if (d->max_depth < 1 || d->max_depth > 16) return SPECA_ERR_RANGE;
     if (d->max_nodes < 1 || d->max_nodes > 1024) return SPECA_ERR_RANGE;
     if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_FACTORIZED) return SPECA_ERR_UNSUPPORTED;
+    if (d->rule != SPECA_RULE_GATED_DELTA && d->rule != SPECA_RULE_GATED_NO_ERASE) return SPECA_ERR_UNSUPPORTED;
     const long long units = 1LL * d->n_layers * d->batch * d->heads;
     if (units * (d->d_v / 2) > 0x7fffffffLL) return SPECA_ERR_RANGE;       // grid size bound
     return SPECA_OK;
@@ -26,6 +27,7 @@ Params base_params(const speca_dims *d, int32_t total_nodes)
     Params p{};
     p.L = d->n_layers; p.B = d->batch; p.H = d->heads; p.T = total_nodes; p.DV = d->d_v;
     p.scale = d->scale; p.max_depth = d->max_depth; p.max_nodes = d->max_nodes;
+    p.no_erase = d->rule == SPECA_RULE_GATED_NO_ERASE;
     return p;
 }
 

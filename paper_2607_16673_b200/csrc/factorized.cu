@@ -967,7 +967,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                 for (int j = kMaxDepth - 2; j >= 0; --j) {
                     const bool is_anc = active && j < d - 1;
-                    c[j] = is_anc ? sgn * ratio * gsel[j] : 0.f;
+                    // without the erase term u_t = beta_t v_t: the key rows contribute nothing but cV
+                    c[j] = (is_anc && !(is_k && p.no_erase)) ? sgn * ratio * gsel[j] : 0.f;
                     if (is_anc) ratio *= anc_alpha[j];
                 }
                 // after the loop ratio = gamma (product of alpha over the whole root path)
@@ -975,7 +976,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     c[7] = active ? -sgn : 0.f;                                       // cV = beta
                     reinterpret_cast<float4 *>(cf)[0] = make_float4(c[0], c[1], c[2], c[3]);
                     reinterpret_cast<float4 *>(cf)[1] = make_float4(c[4], c[5], c[6], c[7]);
-                    cf[16] = active ? sgn * ratio * kDebias : 0.f;                              // cR = -beta gamma
+                    cf[16] = (active && !p.no_erase) ? sgn * ratio * kDebias : 0.f;            // cR = -beta gamma
                 } else {
                     // level d-1 is the node itself: (q_t . k_t) with ratio 1
                     c[7] = 0.f;

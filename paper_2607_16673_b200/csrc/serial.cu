@@ -110,7 +110,7 @@ decode_kernel(Params p)
         const float sk = group_sum<G>(dot16(s[r], kx));
         const float sq = group_sum<G>(dot16(s[r], qx));
         const float vv = bf16_to_float(p.v + unit * p.DV + row);
-        const float u = beta * (vv - alpha * sk);
+        const float u = p.no_erase ? beta * vv : beta * (vv - alpha * sk);
         axpy16(s[r], kx, alpha, u);
         store_row<G>(Su + long(row) * DK, g, s[r]);
         if (g == 0) p.o[unit * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
@@ -185,7 +185,7 @@ verify_serial_kernel(Params p)
             const float sk = group_sum<G>(dot16(s[r], kx));
             const float sq = group_sum<G>(dot16(s[r], qx));
             const float vv = bf16_to_float(p.v + rec * p.DV + row);
-            const float u = beta * (vv - alpha * sk);
+            const float u = p.no_erase ? beta * vv : beta * (vv - alpha * sk);
             if (!leaf) axpy16(s[r], kx, alpha, u);
             if (g == 0) {
                 p.o[rec * p.DV + row] = p.scale * fmaf(alpha, sq, u * kq);
@@ -299,7 +299,7 @@ commit_kernel(Params p)
         for (int r = 0; r < RS; ++r) {
             const float sk = group_sum<G>(dot16(s[r], kx));
             const float vv = __bfloat162float(s_v[d][tile_row + r * RPS]);
-            const float u = beta * (vv - alpha * sk);
+            const float u = p.no_erase ? beta * vv : beta * (vv - alpha * sk);
             axpy16(s[r], kx, alpha, u);
         }
     }

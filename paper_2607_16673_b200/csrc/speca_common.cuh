@@ -73,6 +73,7 @@ struct Params {
     int32_t L, B, H, T, DV;
     float scale;
     int32_t max_depth, max_nodes;
+    int32_t no_erase;            // SPECA_RULE_GATED_NO_ERASE: the corrected value is u = beta v (no read-out of the state)
     float *S;                    // in/out for decode and commit
     const float *S0;             // read-only for verify
     const __nv_bfloat16 *q, *k, *v;

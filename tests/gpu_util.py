@@ -33,13 +33,13 @@ class DevProblem:
     """A synth.Problem resident on the GPU plus output buffers."""
 
     def __init__(self, prob: synth.Problem, route=speca.ROUTE_AUTO, max_nodes=None, want_u=False,
-                 device="cuda"):
+                 device="cuda", rule=0):
         self.prob = prob
         sizes = np.diff(prob.node_offsets)
         if max_nodes is None:
             max_nodes = max(1, int(sizes.max()) if sizes.size else 1)
         self.dims = speca.Dims(prob.L, prob.B, prob.H, prob.d_k, prob.d_v, prob.scale, prob.max_depth,
-                               max_nodes, route)
+                               max_nodes, route, rule)
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
         self.S = t(prob.S0)
         self.q, self.k, self.v = bf16_dev(prob.q, device), bf16_dev(prob.k, device), bf16_dev(prob.v, device)

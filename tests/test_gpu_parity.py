@@ -476,3 +476,43 @@ def test_deltanet_records_are_the_alpha_one_case(route):
     assert rel_err(cpu(S), S_ref) <= tol_for(route) and rel_err(cpu(d2.o), o_ref) <= tol_for(route)
     d1.commit()
     assert rel_err(cpu(d1.S), S_ref) <= TOL_FP32
+
+
+@pytest.mark.parametrize("route", ROUTES)
+def test_rule_without_erase(route):
+    """GLA-style records (key, value, gate; no delta-rule read-out): dims.rule = GATED_NO_ERASE on decode,
+    verify, commit and the fused call, against the oracle set to the same rule."""
+    rng = np.random.default_rng(1001)
+    p1 = synth.make_problem(1002, 2, 4, 128, 256, synth.ragged_tree_batch(rng, 4, 4, 40, 8))
+    p2 = synth.make_problem(1003, 2, 4, 128, 256, synth.ragged_tree_batch(rng, 4, 4, 40, 8))
+    R = speca.RULE_GATED_NO_ERASE
+    try:
+        oracle.set_rule(oracle.RULE_GATED_NO_ERASE)
+        o1_ref = oracle_verify(p1)
+        pi, pl, _ = oracle.greedy_accept(p1.node_offsets, p1.parent, p1.draft_tok, p1.target_tok, p1.root_target_tok, 8)
+        S_ref = oracle_commit(p1, pi, pl)
+        o2_ref = oracle.verify_tree(S_ref, p2.q, p2.k, p2.v, p2.alpha, p2.beta, p2.node_offsets, p2.parent)
+        q1, k1, v1, a1, b1 = synth.draw_records(rng, p1.L, p1.B, p1.H, p1.d_k, p1.d_v)
+        Sd_ref, od_ref = oracle.decode_step(p1.S0, q1, k1, v1, a1, b1)
+    finally:
+        oracle.set_rule(oracle.RULE_GATED_DELTA)
+    d1 = DevProblem(p1, route=route, want_u=True, max_nodes=64, rule=R)
+    d1.verify_tree()
+    assert d1.status_value() == 0 and rel_err(cpu(d1.o), o1_ref) <= tol_for(route)
+    d1.accept()
+    d2 = DevProblem(p2, route=route, want_u=True, max_nodes=64, rule=R)
+    S = d1.S.clone()
+    prev = dict(k=d1.k, v=d1.v, alpha=d1.alpha, beta=d1.beta, u=d1.u, node_offsets=d1.node_offsets, total_nodes=d1.T,
+                parent=d1.parent)
+    speca.commit_verify_tree(d2.dims, S, prev, d1.path_idx, d1.path_len, d2.q, d2.k, d2.v, d2.alpha, d2.beta,
+                             d2.node_offsets, d2.T, d2.parent, None, d2.o, d2.u, d2.ws, d2.status)
+    assert d2.status_value() == 0
+    assert rel_err(cpu(S), S_ref) <= tol_for(route) and rel_err(cpu(d2.o), o2_ref) <= tol_for(route)
+    d1.commit()
+    assert rel_err(cpu(d1.S), S_ref) <= TOL_FP32
+    from gpu_util import bf16_dev
+    Sd = torch.from_numpy(p1.S0).cuda()
+    od = torch.empty(p1.L, p1.B, p1.H, p1.d_v, device="cuda")
+    speca.decode_step(speca.Dims(p1.L, p1.B, p1.H, p1.d_k, p1.d_v, rule=R), Sd, bf16_dev(q1), bf16_dev(k1), bf16_dev(v1),
+                      torch.from_numpy(a1).cuda(), torch.from_numpy(b1).cuda(), od)
+    assert rel_err(cpu(Sd), Sd_ref) <= TOL_FP32 and rel_err(cpu(od), od_ref) <= TOL_FP32

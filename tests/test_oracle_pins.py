@@ -557,6 +557,38 @@ def test_pruning_hand_case_and_selection_properties():
                 assert (par[i] < 0 and newpar[r] == -1) or got[newpar[r]] == par[i]
 
 
+def test_rule_without_erase_is_gated_linear_attention():
+    """Rule 1 (GLA-style records, Section 5.1 remark): S' = alpha S + beta v k^T.  Closed form along a path:
+    S_t = gamma_t S0 + sum_{i on path} (gamma_t / gamma_i) beta_i v_i k_i^T, evaluated directly with numpy for
+    every node of a tree; commit over a path likewise.  The default rule is restored afterwards."""
+    rng = np.random.default_rng(71)
+    par = synth.random_tree_parent(12, 5, 3, rng)
+    prob = synth.make_problem(71, 2, 2, 16, 8, [par])
+    try:
+        oracle.set_rule(oracle.RULE_GATED_NO_ERASE)
+        o = run_verify(prob)
+        path = synth.root_path(par, 11)
+        idx = np.full((1, 8), -1, np.int32); idx[0, :len(path)] = path
+        Sc = oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets, idx,
+                           np.array([len(path)], np.int32))
+    finally:
+        oracle.set_rule(oracle.RULE_GATED_DELTA)
+    for l in range(2):
+        for h in range(2):
+            S0, q, k, v, al, be, _ = unit_arrays(prob, l=l, b=0, h=h)
+            def state(t):
+                pth = synth.root_path(par, t)
+                gam = np.cumprod([al[i] for i in pth])
+                S = gam[-1] * S0
+                for j, i in enumerate(pth):
+                    S = S + (gam[-1] / gam[j]) * be[i] * np.outer(v[i], k[i])
+                return S
+            for t in range(12):
+                assert np.allclose(state(t) @ q[t], o[l, t, h], rtol=1e-12, atol=1e-14)
+            assert np.allclose(state(11), Sc[l, 0, h], rtol=1e-12, atol=1e-14)
+    assert not np.allclose(run_verify(prob), o)          # and it is a different rule from the default one
+
+
 def test_paper_byte_counts():
     vals = {}
     for r in open(os.path.join(GOLDEN, "paper_sizes.txt")):
