@@ -55,14 +55,9 @@ constexpr int kChunkK = 32;                    // floats per 128-byte swizzle ro
 constexpr int kChunks = kDK / kChunkK;         // 4 K-chunks per tile
 constexpr int kStageBytes = kTileRows * 128;   // 16 KiB per (tile, K-chunk)
 constexpr int kStages = 6;
-#ifndef SPECA_POLL_NS
-#define SPECA_POLL_NS 100
-#endif
-#ifndef SPECA_FUSED_STAGES
-#define SPECA_FUSED_STAGES 5
-#endif
-constexpr int kStagesFused = SPECA_FUSED_STAGES;                // the fused kernel reads the state at half its total traffic: a
-                                               // shallower ring suffices, the other two slots hold the pending u rows
+constexpr int kStagesFused = 5;                // the fused kernel's ring: its sixth slot holds the staged u rows of the pending
+                                               // paths (the kernel reads the state at about half of its total traffic)
+constexpr int kPollNs = 100;                   // pause of the fused producer when neither a load nor a store is ready
 constexpr int kMaxNodes = 64;                  // nodes per sequence handled by this route
 constexpr int kMaxDepth = 8;
 constexpr int kBopRows = 2 * kMaxNodes;        // [K;Q] rows
@@ -72,10 +67,7 @@ constexpr int kAccCols = 2 * kMaxNodes;        // 128 TMEM columns per tile accu
 constexpr int kPairCols = 2 * kAccCols;        // a unit's two tiles
 constexpr int kTmemCols = 512;                 // two units in flight
 constexpr int kThreads = 14 * 32;
-#ifndef SPECA_UPD_WARPS
-#define SPECA_UPD_WARPS 2
-#endif
-constexpr int kUpdWarps = SPECA_UPD_WARPS;                   // state-update role of the fused kernel
+constexpr int kUpdWarps = 2;                   // state-update role of the fused kernel
 constexpr int kUpdThreads = kUpdWarps * 32;
 constexpr int kThreadsFused = kThreads + kUpdThreads;
 constexpr int kPrepThreads = 128;
@@ -104,9 +96,9 @@ constexpr int kOffPendK = kOffMisc + 64;                                  // bf1
 constexpr int kKeyStride = kDK * 2 + 16;                                   // bytes per staged pending key (bank padding)
 constexpr int kKeyBuf = kMaxDepth * kKeyStride;
 constexpr int kOffWalk = kOffPendK + 2 * kKeyBuf;                          // per-sequence walk table
-// fused kernel: u rows of the pending path, [2][8][256 + 16] fp32, in ring slots 4 and 5
+// fused kernel: u rows of the pending path, [2][8][256] fp32, in the sixth ring slot
 constexpr int kOffPendU = kOffRing + kStagesFused * kStageBytes;
-constexpr int kPendUStride = (2 * kTileRows + (kStagesFused <= 4 ? 16 : 0)) * 4;
+constexpr int kPendUStride = 2 * kTileRows * 4;
 constexpr int kPendUBuf = kMaxDepth * kPendUStride;
 static_assert(2 * kPendUBuf <= (kStages - kStagesFused) * kStageBytes, "pending u rows do not fit the spare ring slots");
 constexpr int kWalkSeqs = 192;                                            // sequences the table holds
@@ -668,7 +660,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     for (uint32_t spin = 0; ok; ++spin) {
                         if (__all_sync(0xffffffffu, mbar_test_wait(be, pe))) break;
                         if (ist < it && updated(ist, false) == 1) issue_store();
-                        else __nanosleep(SPECA_POLL_NS);         // nothing to do: leave the issue slots to the other warps
+                        else __nanosleep(kPollNs);         // nothing to do: leave the issue slots to the other warps
                         if ((spin & 255u) == 255u) {
                             if (__any_sync(0xffffffffu, *abort_flag != 0)) ok = false;
                             const uint64_t now = global_timer_ns();
