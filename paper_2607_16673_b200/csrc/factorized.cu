@@ -363,6 +363,12 @@ __device__ __forceinline__ int anc_byte(const int4 &meta, int j)
 {
     return int((j < 4 ? (uint32_t(meta.y) >> (8 * j)) : (uint32_t(meta.z) >> (8 * (j - 4)))) & 0xffu);
 }
+// levels 0..14 (trees up to 16 deep): levels 8..11 in the first record's last word, 12..14 in the second record
+__device__ __forceinline__ int anc_byte16(const int4 &meta, int meta2, int j)
+{
+    const uint32_t w = j < 4 ? uint32_t(meta.y) : j < 8 ? uint32_t(meta.z) : j < 12 ? uint32_t(meta.w) : uint32_t(meta2);
+    return int((w >> (8 * (j & 3))) & 0xffu);
+}
 
 // kind::f16 with bf16 operands, fp32 accumulate, both operands K-major, M = 128 (Gram block)
 __device__ __forceinline__ uint32_t make_idesc_bf16(int n)
@@ -479,10 +485,51 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
     }
 }
 
+// The same step for trees up to MAXD levels deep (the coefficient record is cU[MAXD-1] cV cO[MAXD] cR cG
+// depth-1 offset).  Used for MAXD = 16; the 8-level form above is kept as it is because the shape of its
+// two accumulation chains was tuned.
+template <int TP, int MAXD>
+__device__ __forceinline__ void node_step_deep(float (&ustk)[TP][MAXD], const float *cf, const float (&Rv)[TP],
+                                               const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
+                                               float (&o_out)[TP], int &off)
+{
+    float cu[MAXD], co[MAXD];
+#pragma unroll
+    for (int i = 0; i < MAXD / 4; ++i) {
+        const float4 a = *reinterpret_cast<const float4 *>(cf + 4 * i), b = *reinterpret_cast<const float4 *>(cf + MAXD + 4 * i);
+        cu[4 * i] = a.x; cu[4 * i + 1] = a.y; cu[4 * i + 2] = a.z; cu[4 * i + 3] = a.w;
+        co[4 * i] = b.x; co[4 * i + 1] = b.y; co[4 * i + 2] = b.z; co[4 * i + 3] = b.w;
+    }
+    const float4 s = *reinterpret_cast<const float4 *>(cf + 2 * MAXD);
+    const int d1 = __float_as_int(s.z);
+    off = __float_as_int(s.w);
+#pragma unroll
+    for (int t = 0; t < TP; ++t) {
+        float u0 = fmaf(cu[MAXD - 1], vv[t], s.x * Rv[t]), u1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < MAXD - 1; ++j) {
+            if (j & 1) u1 = fmaf(cu[j], ustk[t][j], u1);
+            else u0 = fmaf(cu[j], ustk[t][j], u0);
+        }
+        const float u = u0 + u1;
+#pragma unroll
+        for (int j = 0; j < MAXD; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        float o0 = s.y * Gv[t], o1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < MAXD; ++j) {
+            if (j & 1) o1 = fmaf(co[j], ustk[t][j], o1);
+            else o0 = fmaf(co[j], ustk[t][j], o0);
+        }
+        o_out[t] = o0 + o1;
+        u_out[t] = u;
+    }
+}
+
 // TP = value tiles per unit (d_v / 128): 1 or 2.  FUSED adds the state-update role (d_k = 128 only).
 // DK = key width, 128 or 256.  The operand buffers have a fixed size, so the wider key halves
 // the number of [K;Q] rows they hold: up to 64 nodes per sequence at d_k = 128, 32 at d_k = 256.
-template <int TP, bool FUSED, int DK = kDK>
+// DEEP: trees up to 16 levels deep (up to 32 nodes per sequence at either key width; not with FUSED).
+template <int TP, bool FUSED, int DK = kDK, bool DEEP = false>
 __global__ void __launch_bounds__(FUSED ? kThreadsFused : kThreads, 1)
 verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
@@ -552,7 +599,11 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     constexpr int SC = DK / 64;                                   // 64-column chunks of the staged bf16 rows
     constexpr int SCB = BROWS * 128;                              // bytes of one such chunk
     static_assert(NC * BCB == kChunks * kBopChunkBytes && SC * SCB == 2 * kStageChunkBytes, "operand buffers keep their size");
-    constexpr int MAXN = BROWS / 2;                               // nodes per sequence; also the stride of the coefficient buffers
+    static_assert(!(FUSED && DEEP), "the fused kernel takes pending paths and trees of at most 8 levels");
+    constexpr int MAXD = DEEP ? 2 * kMaxDepth : kMaxDepth;        // tree depth this instantiation takes
+    constexpr int CS = 2 * MAXD + 4;                              // floats of a coefficient record
+    constexpr int MAXN = DEEP ? kMaxNodes / 2 : BROWS / 2;        // nodes per sequence; also the stride of the coefficient buffers
+    static_assert(2 * MAXN * CS * 4 <= 2 * kMaxNodes * kCoefStride * 4 && CS % 4 == 0, "coefficient records do not fit");
     // Fused kernel: staged bf16 keys of the pending path, two buffers of 8 padded rows.  At d_k = 128 both
     // sit in their own region; at d_k = 256 a buffer is twice as large, and the second one takes the half
     // of the coefficient region that 32-node sequences leave unused.
@@ -560,7 +611,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     static_assert(DK == kDK ? 2 * KBUF <= kOffWalk - kOffPendK
                             : (KBUF <= kOffWalk - kOffPendK && KBUF <= kMaxNodes * kCoefStride * 4), "pending keys do not fit");
     auto key_buf = [](int pb) -> int {
-        return DK == kDK ? kOffPendK + pb * KBUF : (pb == 0 ? kOffPendK : kOffCoef + 2 * MAXN * kCoefStride * 4);
+        return DK == kDK ? kOffPendK + pb * KBUF : (pb == 0 ? kOffPendK : kOffCoef + 2 * MAXN * CS * 4);
     };
     UnitWalk walk;
     walk.HG = fp.heads_per_group; walk.gpl = p.H / fp.heads_per_group;
@@ -815,6 +866,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         unsigned long long node_lo = ~0ull, node_hi = ~0ull;   // node at the position of each handled row (0xff = none)
         int topo_grp = -1;
         int4 meta_nxt = make_int4(0, 0, 0, 0);
+        int meta2_nxt = 0;                                       // DEEP: ancestors of levels 12..14
         // start the TMA copies of unit x's rows (one thread), fetch alpha / beta and, when the
         // sequence changes, the topology this thread needs
         auto prefetch = [&](const Unit &x) {
@@ -843,6 +895,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 const int node = row < x.npad ? row : row - x.npad;
                 meta_nxt = (row < 2 * x.npad && node < x.n)
                                ? __ldg(reinterpret_cast<const int4 *>(p.ws.anc) + x.base + node) : make_int4(0, 0, 0, 0);
+                if (DEEP) meta2_nxt = (row < 2 * x.npad && node < x.n) ? __ldg(p.ws.anc2 + 4 * (x.base + node)) : 0;
             }
             if (tid < x.n) {
                 const int rec = (x.l * p.T + x.base + tid) * p.H + x.h;
@@ -857,6 +910,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         bool have = first_unit(walk, x);
         if (have) prefetch(x);
         int4 meta = meta_nxt;
+        int meta2 = meta2_nxt;
         unsigned long long cur_lo = node_lo, cur_hi = node_hi;
         PROF_DECL
         for (; have && ok; ++unit_seq) {
@@ -911,16 +965,17 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             const int d = meta.x & 0xff;
             const int pos = active ? ((meta.x >> 8) & 0xff) : node;       // padding rows: any unused record (n <= node < npad)
             // ancestors by level (level d-1 is the node itself), their alpha, and this row's Gram entries
-            int anc_pos[kMaxDepth];
-            float anc_alpha[kMaxDepth], gsel[kMaxDepth];
+            int anc_pos[MAXD];
+            float anc_alpha[MAXD], gsel[MAXD];
 #pragma unroll
-            for (int j = 0; j < kMaxDepth; ++j) anc_pos[j] = !active ? 0 : ((j < d - 1) ? anc_byte(meta, j) : node);
+            for (int j = 0; j < MAXD; ++j)
+                anc_pos[j] = !active ? 0 : ((j < d - 1) ? (DEEP ? anc_byte16(meta, meta2, j) : anc_byte(meta, j)) : node);
 
             // park this thread's Gram row in its private scratch column (32 columns per pass),
             // then pick the entries it needs
             const uint32_t gaddr = tmem_base + par * kPairCols + lane_addr;
 #pragma unroll
-            for (int j = 0; j < kMaxDepth; ++j) gsel[j] = 0.f;
+            for (int j = 0; j < MAXD; ++j) gsel[j] = 0.f;
 #pragma unroll 1
             for (int half = 0; half * kGramHalf < x.npad; ++half) {
 #pragma unroll 1
@@ -935,7 +990,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     for (int i = 0; i < 8; ++i) gram[(c0 + 8 + i) * kTileRows + row] = g1[i];
                 }
 #pragma unroll
-                for (int j = 0; j < kMaxDepth; ++j)
+                for (int j = 0; j < MAXD; ++j)
                     if ((anc_pos[j] >> 5) == half) gsel[j] = gram[(anc_pos[j] & 31) * kTileRows + row];
             }
             tc_fence_before();
@@ -945,7 +1000,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             // doubles as the prep-internal barrier)
             if (!(ok = WAIT(3, bar(kBarBReady), unit_seq & 1))) break;
 #pragma unroll
-            for (int j = 0; j < kMaxDepth; ++j) anc_alpha[j] = alpha_s[anc_pos[j]];
+            for (int j = 0; j < MAXD; ++j) anc_alpha[j] = alpha_s[anc_pos[j]];
             const float my_a = alpha_s[active ? node : 0];
             const float sgn = is_k ? -beta_s[active ? node : 0] : p.scale;
             // the coefficient buffer of this parity must have been released by the epilogue
@@ -953,33 +1008,36 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             // coefficient record of this row's node; levels that are not ancestors stay zero, rows
             // past the last node (padding up to a multiple of 16) become no-op records
             if (in_rows) {
-                float *cf = reinterpret_cast<float *>(smem + kOffCoef) + (par * MAXN + pos) * kCoefStride;
-                float c[kMaxDepth];
+                float *cf = reinterpret_cast<float *>(smem + kOffCoef) + (par * MAXN + pos) * CS;
+                float c[MAXD];
                 float ratio = my_a;
 #pragma unroll
-                for (int j = kMaxDepth - 2; j >= 0; --j) {
+                for (int j = MAXD - 2; j >= 0; --j) {
                     const bool is_anc = active && j < d - 1;
                     // without the erase term u_t = beta_t v_t: the key rows contribute nothing but cV
                     c[j] = (is_anc && !(is_k && p.no_erase)) ? sgn * ratio * gsel[j] : 0.f;
                     if (is_anc) ratio *= anc_alpha[j];
                 }
                 // after the loop ratio = gamma (product of alpha over the whole root path)
+                // record: cU[MAXD-1] cV | cO[MAXD] | cR cG depth-1 offset
                 if (is_k) {
-                    c[7] = active ? -sgn : 0.f;                                       // cV = beta
-                    reinterpret_cast<float4 *>(cf)[0] = make_float4(c[0], c[1], c[2], c[3]);
-                    reinterpret_cast<float4 *>(cf)[1] = make_float4(c[4], c[5], c[6], c[7]);
-                    cf[16] = (active && !p.no_erase) ? sgn * ratio * kDebias : 0.f;            // cR = -beta gamma
+                    c[MAXD - 1] = active ? -sgn : 0.f;                                // cV = beta
+#pragma unroll
+                    for (int i = 0; i < MAXD / 4; ++i)
+                        reinterpret_cast<float4 *>(cf)[i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
+                    cf[2 * MAXD] = (active && !p.no_erase) ? sgn * ratio * kDebias : 0.f;      // cR = -beta gamma
                 } else {
                     // level d-1 is the node itself: (q_t . k_t) with ratio 1
-                    c[7] = 0.f;
+                    c[MAXD - 1] = 0.f;
 #pragma unroll
-                    for (int j = 0; j < kMaxDepth; ++j)
+                    for (int j = 0; j < MAXD; ++j)
                         if (active && j == d - 1) c[j] = sgn * gsel[j];
-                    reinterpret_cast<float4 *>(cf)[2] = make_float4(c[0], c[1], c[2], c[3]);
-                    reinterpret_cast<float4 *>(cf)[3] = make_float4(c[4], c[5], c[6], c[7]);
-                    cf[17] = active ? sgn * ratio * kDebias : 0.f;                              // cG = scale gamma
-                    cf[18] = __int_as_float(active ? d - 1 : -1);
-                    cf[19] = __int_as_float(active ? node * p.H * p.DV : 0);          // offset of the node's row
+#pragma unroll
+                    for (int i = 0; i < MAXD / 4; ++i)
+                        reinterpret_cast<float4 *>(cf)[MAXD / 4 + i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
+                    cf[2 * MAXD + 1] = active ? sgn * ratio * kDebias : 0.f;                  // cG = scale gamma
+                    cf[2 * MAXD + 2] = __int_as_float(active ? d - 1 : -1);
+                    cf[2 * MAXD + 3] = __int_as_float(active ? node * p.H * p.DV : 0);        // offset of the node's row
                 }
             }
             mbar_arrive(bar(kBarCoefReady + par));
@@ -993,6 +1051,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             x = nx;
             have = have_next;
             meta = meta_nxt;
+            meta2 = meta2_nxt;
             cur_lo = node_lo; cur_hi = node_hi;
         }
         PROF_STORE()
@@ -1002,7 +1061,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         const int row = 32 * (warp & 3) + lane;
         const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
         const uint32_t acc = tmem_base + grp * kPairCols + lane_addr;
-        const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * MAXN * kCoefStride;
+        const float *coef = reinterpret_cast<const float *>(smem + kOffCoef) + grp * MAXN * CS;
 
         // this group's units: unit_seq == grp (mod 2)
         Unit x;
@@ -1042,11 +1101,11 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             const VPack *v_row = vraw + rec0 * kTileRows + row;
             float *o_row = p.o + rec0 * p.DV + row * TP;
             float *u_row = p.u != nullptr ? p.u + rec0 * p.DV + row * TP : nullptr;
-            float ustk[TP][kMaxDepth];
+            float ustk[TP][MAXD];
 #pragma unroll
             for (int t = 0; t < TP; ++t)
 #pragma unroll
-                for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = 0.f;
+                for (int j = 0; j < MAXD; ++j) ustk[t][j] = 0.f;
             const int npad = x.npad, n = x.n;
             auto load_tmem = [&](int p0, float (&R)[TP][kEpiChunk], float (&G)[TP][kEpiChunk]) {
 #pragma unroll
@@ -1058,7 +1117,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             auto load_values = [&](int p0, VPack (&vv)[kEpiChunk]) {
 #pragma unroll
                 for (int i = 0; i < kEpiChunk; ++i) {
-                    const int off = __float_as_int(coef[(p0 + i) * kCoefStride + 19]);   // p0 + i < npad; in floats of o
+                    const int off = __float_as_int(coef[(p0 + i) * CS + CS - 1]);        // p0 + i < npad; in floats of o
                     vv[i] = __ldg(v_row + off / TP);
                 }
                 // the value rows of the chunk after this one: into L1 now, so that their loads are short
@@ -1066,7 +1125,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 if (p0 + kEpiChunk < n) {
 #pragma unroll
                     for (int i = 0; i < kEpiChunk; ++i) {
-                        const int offn = __float_as_int(coef[(p0 + kEpiChunk + i) * kCoefStride + 19]);
+                        const int offn = __float_as_int(coef[(p0 + kEpiChunk + i) * CS + CS - 1]);
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(v_row + offn / TP));
                     }
                 }
@@ -1087,7 +1146,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     } else {
                         v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
                     }
-                    node_step<TP>(ustk, coef + (p0 + i) * kCoefStride, r_, g_, v_, uo, oo, off);
+                    if constexpr (DEEP) node_step_deep<TP, MAXD>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
+                    else node_step<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
                     if (p0 + i < n) {
                         if (TP == 2) {
                             *reinterpret_cast<float2 *>(o_row + off) = make_float2(oo[0], oo[TP - 1]);
@@ -1307,11 +1367,14 @@ EncodeTiledFn encode_tiled_fn()
 
 bool factorized_supported(const speca_dims *d)
 {
-    const bool keys = (d->d_k == kDK && d->max_nodes <= kMaxNodes) || (d->d_k == 2 * kDK && d->max_nodes <= kMaxNodes / 2);
-    return keys && (d->d_v == kTileRows || d->d_v == 2 * kTileRows) && d->max_depth <= kMaxDepth;
+    if (d->d_k != kDK && d->d_k != 2 * kDK) return false;
+    if (d->d_v != kTileRows && d->d_v != 2 * kTileRows) return false;
+    // trees of at most 8 levels: 64 nodes per sequence at d_k = 128, 32 at d_k = 256; up to 16 levels: 32 nodes
+    if (d->max_depth <= kMaxDepth) return d->max_nodes <= (d->d_k == kDK ? kMaxNodes : kMaxNodes / 2);
+    return d->max_depth <= 2 * kMaxDepth && d->max_nodes <= kMaxNodes / 2;
 }
 
-bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d); }
+bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d) && d->max_depth <= kMaxDepth; }
 
 int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st)
 {
@@ -1371,7 +1434,11 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
             reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256>),
             reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256>),
             reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 256>)};
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 256>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 128, true>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 128, true>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256, true>),
+            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256, true>)};
         for (const void *k : kernels) {
             cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
             if (e != cudaSuccess) return int(e);
@@ -1395,6 +1462,14 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
     } else if (fused) {
         if (one_tile) verify_factorized_kernel<1, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
         else verify_factorized_kernel<2, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
+    } else if (p.max_depth > kMaxDepth) {
+        if (d_k == kDK) {
+            if (one_tile) verify_factorized_kernel<1, false, 128, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+            else verify_factorized_kernel<2, false, 128, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        } else {
+            if (one_tile) verify_factorized_kernel<1, false, 256, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+            else verify_factorized_kernel<2, false, 256, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
+        }
     } else if (d_k == kDK) {
         if (one_tile) verify_factorized_kernel<1, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
         else verify_factorized_kernel<2, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);

@@ -112,25 +112,27 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
     }
     __syncthreads();
     // Per node: depth, position in the processing order, and the node's ancestors by depth
-    // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 8, which is all
-    // the factorised route accepts).
+    // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 16, which is all
+    // the factorised route accepts).  Level j (0 = child of the committed state) of the first
+    // record sits in byte j % 4 of word 1 + j / 4 for j < 12; levels 12..14 are in the second.
     for (int i = tid; i < n; i += kPlanThreads) {
         int d = 0;
         for (int a = i; a >= 0; a = par[a]) ++d;
-        uint32_t lo = 0, hi = 0;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
         int j = d - 1;
         for (int a = par[i]; a >= 0; a = par[a]) {
             --j;
-            const uint32_t byte = uint32_t(a) & 0xffu;
-            if (j < 4) lo |= byte << (8 * j);
-            else if (j < 8) hi |= byte << (8 * (j - 4));
+            if (j < 16) w[j >> 2] |= (uint32_t(a) & 0xffu) << (8 * (j & 3));
         }
-        int4 rec;
+        int4 rec, rec2;
         rec.x = d | (posn[i] << 8);
-        rec.y = int(lo);
-        rec.z = int(hi);
-        rec.w = 0;
+        rec.y = int(w[0]);
+        rec.z = int(w[1]);
+        rec.w = int(w[2]);
+        rec2.x = int(w[3]);
+        rec2.y = rec2.z = rec2.w = 0;
         reinterpret_cast<int4 *>(ws.anc)[base + i] = rec;
+        reinterpret_cast<int4 *>(ws.anc2)[base + i] = rec2;
     }
     __syncthreads();
     if (tid == 0) {

@@ -15,7 +15,7 @@ namespace speca {
 //   [0, 2048)                    control words (work-queue counters, optional profiling slots)
 //   [2048, 2048 + 4*Bpad)        seq_n[b]: node count of sequence b, or -1 if the
 //                                sequence failed validation and must be skipped
-//   then int32 arrays of Tpad words: plan[T], depth[T], anc[T][4]
+//   then int32 arrays of Tpad words: plan[T], depth[T], anc[T][4], anc2[T][4]
 //   after the kNodeWords node arrays, used only by the fused commit-and-verify call:
 //   pend[B][kPendWords]: validated length of the pending accepted path, its local node
 //   indices, and the sequence's offset in the previous draft's packed arrays
@@ -32,7 +32,8 @@ struct Workspace {
     int32_t *seq_n;     // [B]
     int32_t *plan;      // [T]   packed schedule entries, in processing order per sequence
     int32_t *depth;     // [T]   depth computed from parent[]
-    int32_t *anc;       // [T][4] per node: depth | position << 8, ancestor node indices by level (8 bytes), spare
+    int32_t *anc;       // [T][4] per node: depth | position << 8, ancestor node indices of levels 1..12 (one byte each)
+    int32_t *anc2;      // [T][4] per node: ancestor node indices of levels 13..15, spare
     int32_t *pend;      // [B][kPendWords] pending accepted path (fused commit-and-verify only)
 };
 
@@ -54,6 +55,7 @@ inline Workspace carve_workspace(void *base, int32_t batch, int32_t total_nodes)
     w.plan = reinterpret_cast<int32_t *>(p);
     w.depth = reinterpret_cast<int32_t *>(p + tb);
     w.anc = reinterpret_cast<int32_t *>(p + 2 * tb);
+    w.anc2 = reinterpret_cast<int32_t *>(p + 6 * tb);
     w.pend = reinterpret_cast<int32_t *>(p + kNodeWords * tb);
     return w;
 }

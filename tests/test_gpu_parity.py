@@ -516,3 +516,56 @@ def test_rule_without_erase(route):
     speca.decode_step(speca.Dims(p1.L, p1.B, p1.H, p1.d_k, p1.d_v, rule=R), Sd, bf16_dev(q1), bf16_dev(k1), bf16_dev(v1),
                       torch.from_numpy(a1).cuda(), torch.from_numpy(b1).cuda(), od)
     assert rel_err(cpu(Sd), Sd_ref) <= TOL_FP32 and rel_err(cpu(od), od_ref) <= TOL_FP32
+
+
+@pytest.mark.parametrize("d_k,d_v", [(128, 128), (128, 256), (256, 128), (256, 256)])
+def test_factorized_deep_trees(d_k, d_v):
+    """Trees 9 to 16 levels deep (the paper's top-2 proposal shapes) on the tensor-core route: up to 32 nodes."""
+    rng = np.random.default_rng(1100 + d_k + d_v)
+    parents = [synth.proposal_tree_parent(2, 12, 16, rng), synth.proposal_tree_parent(2, 24, 32, rng),
+               synth.proposal_tree_parent(4, 12, 16, rng), synth.chain_parent(16), np.zeros(0, np.int32),
+               synth.random_tree_parent(32, 16, 3, rng), synth.chain_parent(1), synth.random_tree_parent(20, 5, 3, rng),
+               synth.chain_parent(9)]
+    prob = synth.make_problem(1101 + d_k + d_v, 2, 4, d_k, d_v, parents, max_depth=16, name=f"deep-{d_k}x{d_v}")
+    assert int(prob.depth.max()) == 16
+    dp, ref = check_verify(prob, speca.ROUTE_FACTORIZED, want_u=True, max_nodes=32)
+    ds = DevProblem(prob, route=speca.ROUTE_SERIAL, want_u=True, max_nodes=32)
+    ds.verify_tree()
+    assert rel_err(cpu(dp.o), cpu(ds.o)) <= TOL and rel_err(cpu(dp.u), cpu(ds.u)) <= TOL
+    # paths up to 16 nodes long: accept and commit (fp32 kernel)
+    dp.accept()
+    pi, pl, _ = oracle.greedy_accept(prob.node_offsets, prob.parent, prob.draft_tok, prob.target_tok,
+                                     prob.root_target_tok, prob.max_depth)
+    assert np.array_equal(cpu(dp.path_idx), pi) and np.array_equal(cpu(dp.path_len), pl)
+    dp.commit()
+    assert rel_err(cpu(dp.S), oracle_commit(prob, pi, pl)) <= TOL_FP32
+    # 33 nodes at this depth is outside the route
+    big = synth.make_problem(1102, 1, 2, d_k, d_v, [synth.random_tree_parent(33, 12, 3, rng)], max_depth=16)
+    with pytest.raises(speca.SpecaError, match="unsupported"):
+        DevProblem(big, route=speca.ROUTE_FACTORIZED, max_nodes=33).verify_tree()
+    check_verify(big, speca.ROUTE_AUTO, tol=TOL_FP32, max_nodes=33)
+
+
+def test_fused_call_with_deep_trees_takes_the_two_kernel_path():
+    rng = np.random.default_rng(1200)
+    mk = lambda seed: synth.make_problem(seed, 2, 4, 128, 256, [synth.proposal_tree_parent(2, 12, 16, rng), synth.chain_parent(12),
+                                                                 synth.random_tree_parent(30, 14, 3, rng)], max_depth=16)
+    p1, p2 = mk(1201), mk(1202)
+    paths = [synth.root_path(p1.parent[int(p1.node_offsets[b]):int(p1.node_offsets[b + 1])],
+                             int(np.argmax(p1.depth[int(p1.node_offsets[b]):int(p1.node_offsets[b + 1])]))) for b in range(3)]
+    idx = np.full((3, 16), -1, np.int32); ln = np.zeros(3, np.int32)
+    for b, pth in enumerate(paths):
+        idx[b, :len(pth)] = pth; ln[b] = len(pth)
+    p1.path_idx, p1.path_len = idx, ln
+    d1 = DevProblem(p1, route=speca.ROUTE_AUTO, want_u=True, max_nodes=32)
+    d1.verify_tree()
+    d2 = DevProblem(p2, route=speca.ROUTE_AUTO, want_u=True, max_nodes=32)
+    S = d1.S.clone()
+    prev = dict(k=d1.k, v=d1.v, alpha=d1.alpha, beta=d1.beta, u=d1.u, node_offsets=d1.node_offsets, total_nodes=d1.T,
+                parent=d1.parent)
+    speca.commit_verify_tree(d2.dims, S, prev, d1.path_idx, d1.path_len, d2.q, d2.k, d2.v, d2.alpha, d2.beta,
+                             d2.node_offsets, d2.T, d2.parent, None, d2.o, d2.u, d2.ws, d2.status)
+    assert d2.status_value() == 0
+    S_ref = oracle_commit(p1, idx, ln)
+    o_ref = oracle.verify_tree(S_ref, p2.q, p2.k, p2.v, p2.alpha, p2.beta, p2.node_offsets, p2.parent)
+    assert rel_err(cpu(S), S_ref) <= TOL_FP32 and rel_err(cpu(d2.o), o_ref) <= TOL
