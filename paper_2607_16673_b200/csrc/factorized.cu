@@ -142,11 +142,6 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -231,13 +226,6 @@ __device__ __forceinline__ bool prof_wait(long long &acc, uint32_t bar, uint32_t
 #define PROF_STORE()
 #endif
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
 {
     asm volatile(
@@ -631,7 +619,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         // Stores are committed one bulk group per slice (an empty group for slices of units with
         // nothing pending), so group age equals slice age.
         uint32_t it = 0, ist = 0, pseq = 0;                      // slices loaded, slices stored, staged units
-        Unit x, nx, xs;                                          // unit being loaded, the one after it, unit being stored
+        Unit x, nx, xs = {};                                     // unit being loaded, the one after it, unit being stored
         int js = 0;                                              // slice of xs the store cursor is at
         bool ok = true;
         auto stage_pending = [&](const Unit &y) -> bool {
