@@ -86,6 +86,9 @@ extern "C" {
 #define SPECA_ROUTE_AUTO        0   /* library picks                                              */
 #define SPECA_ROUTE_SERIAL      1   /* state-resident walk, one rank-1 update per node (Section 4.1) */
 #define SPECA_ROUTE_FACTORIZED  2   /* tree-masked WY form on tensor cores (Section 4.2)           */
+/* The tensor-core route takes d_v in {128, 256} and: max_depth <= 8 with max_nodes <= 64 (d_k = 128) or <= 32
+ * (d_k = 256); 8 < max_depth <= 16 with max_nodes <= 32 (d_k = 128 or 256).  AUTO uses it whenever it applies
+ * and the serial route otherwise; asking for it explicitly outside these shapes is SPECA_ERR_UNSUPPORTED. */
 
 /* recurrences (dims.rule; Section 5.1, remark on other layer types).  A DeltaNet layer (k, v, beta, no
  * decay) is the gated delta rule with alpha = 1 and needs no value of its own. */
@@ -195,9 +198,9 @@ int speca_commit(const speca_dims *dims, float *S,
  * u_or_null to be able to fuse the next round; it must not be the buffer u_prev_or_null
  * points to, and o / u must not alias any input.
  *
- * The single-pass kernel runs when the tensor-core route applies (d_k = 128, d_v in
- * {128, 256}, max_nodes <= 64, max_depth <= 8, route != SERIAL) and u_prev_or_null is
- * given: the pending update is then S <- gamma_A S + sum_i (gamma_A / gamma_i) u_i k_i^T,
+ * The single-pass kernel runs when the tensor-core route applies with max_depth <= 8
+ * (d_v in {128, 256}; d_k = 128 with max_nodes <= 64 or d_k = 256 with max_nodes <= 32;
+ * route != SERIAL) and u_prev_or_null is given: the pending update is then S <- gamma_A S + sum_i (gamma_A / gamma_i) u_i k_i^T,
  * which needs only u, k and alpha of the accepted nodes (v_prev and beta_prev are not
  * read).  Otherwise the commit and verify kernels are launched back to back on `stream`
  * with the same results.  workspace_bytes must be at least speca_workspace_bytes(). */
