@@ -41,6 +41,8 @@
 // of three times.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include <type_traits>
 
 #include "speca_common.cuh"
@@ -344,6 +346,7 @@ struct KQMaps { CUtensorMap k[4], q[4], v[4]; };
 struct FParams {
     Params p;
     int32_t heads_per_group;     // consecutive heads of one (layer, sequence) a CTA takes together
+    int32_t withhold_first_load; // test hook: CTA 0 never issues its first state load, so that its waits run out
     long n_units;
 };
 
@@ -746,7 +749,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
-                    if (lane == 0) {
+                    if (lane == 0 && !(fp.withhold_first_load && blockIdx.x == 0 && it == 0)) {
                         mbar_arrive_expect_tx(bar(kBarFull + s), kStageBytes);
                         tma_load_3d(sbase + kOffRing + s * kStageBytes, &s0_map, c * kChunkK, t, row, bar(kBarFull + s));
                     }
@@ -1436,6 +1439,10 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
     FParams fp;
     fp.p = p;
     fp.n_units = n_units;
+    // Failure-detection test hook (plain verification only): with SPECA_TEST_WITHHOLD_FIRST_LOAD=1 in the environment one
+    // CTA's first state slice never arrives; its bounded waits expire, it reports SPECA_STATUS_TIMEOUT and exits cleanly.
+    const char *hook = getenv("SPECA_TEST_WITHHOLD_FIRST_LOAD");
+    fp.withhold_first_load = (hook != nullptr && hook[0] == '1') ? 1 : 0;
     // consecutive heads of one (layer, sequence) a CTA takes together: as many as divide H while
     // every SM still gets a group
     fp.heads_per_group = 1;

@@ -251,3 +251,33 @@ def test_more_sequences_than_the_walk_table_holds():
     assert rel_err(cpu(d1.o), o1_ref) <= TOL
     assert rel_err(cpu(d2.o), o_ref) <= TOL
     assert rel_err(cpu(S), S_ref) <= TOL
+
+
+def _banded(t, pad=256, fill=7.5):
+    """A copy of tensor t placed in the middle of a larger buffer filled with a sentinel."""
+    flat = torch.full((t.numel() + 2 * pad,), fill, dtype=t.dtype, device=t.device)
+    flat[pad:pad + t.numel()] = t.flatten()
+    return flat, flat[pad:pad + t.numel()].view_as(t)
+
+
+def test_tensor_core_kernels_write_nothing_outside_their_tensors():
+    """Guard bands around everything the tensor-core kernels write (o, u, and S for the fused call, which goes
+    back through TMA stores): the sentinel values on both sides must survive."""
+    rng = np.random.default_rng(19)
+    p1 = synth.make_problem(191, 2, 3, 128, 256, synth.ragged_tree_batch(rng, 3, 5, 40, 8))
+    p2 = synth.make_problem(192, 2, 3, 128, 256, synth.ragged_tree_batch(rng, 3, 5, 40, 8))
+    random_paths(rng, p1, zero_frac=0.0)
+    d1 = DevProblem(p1, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    bo, d1.o = _banded(d1.o)
+    bu, d1.u = _banded(d1.u)
+    d1.verify_tree()
+    d2 = DevProblem(p2, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    bo2, d2.o = _banded(d2.o)
+    bu2, d2.u = _banded(d2.u)
+    bS, S = _banded(d1.S)
+    fused_call(d2, S, prev_dict(d1), d1.path_idx, d1.path_len)
+    assert d1.status_value() == 0 and d2.status_value() == 0
+    for band in (bo, bu, bo2, bu2, bS):
+        assert torch.all(band[:256] == 7.5) and torch.all(band[-256:] == 7.5)
+    S_ref, o_ref = oracle_commit_then_verify(p1.S0, p1, p2)
+    assert rel_err(cpu(S), S_ref) <= TOL and rel_err(cpu(d2.o), o_ref) <= TOL

@@ -569,3 +569,21 @@ def test_fused_call_with_deep_trees_takes_the_two_kernel_path():
     S_ref = oracle_commit(p1, idx, ln)
     o_ref = oracle.verify_tree(S_ref, p2.q, p2.k, p2.v, p2.alpha, p2.beta, p2.node_offsets, p2.parent)
     assert rel_err(cpu(S), S_ref) <= TOL_FP32 and rel_err(cpu(d2.o), o_ref) <= TOL
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable(monkeypatch):
+    """Failure detection: every device-side wait is bounded.  With the library's test hook one CTA's first
+    state slice is never requested; its waits run out (2 s), the kernel returns, the status word carries
+    TIMEOUT, and the next call on the same context works."""
+    rng = np.random.default_rng(1300)
+    prob = synth.make_problem(1301, 2, 4, 128, 128, synth.ragged_tree_batch(rng, 3, 4, 20, 8))
+    dp = DevProblem(prob, route=speca.ROUTE_FACTORIZED, max_nodes=64)
+    monkeypatch.setenv("SPECA_TEST_WITHHOLD_FIRST_LOAD", "1")
+    dp.verify_tree()
+    assert dp.status_value() & speca.STATUS_TIMEOUT
+    monkeypatch.delenv("SPECA_TEST_WITHHOLD_FIRST_LOAD")
+    dp.status.zero_()
+    dp.o.fill_(float("nan"))
+    dp.verify_tree()
+    assert dp.status_value() == 0
+    assert rel_err(cpu(dp.o), oracle_verify(prob)) <= TOL
