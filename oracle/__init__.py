@@ -7,6 +7,16 @@ the CUDA library and never imports it.
 The arithmetic lives in ``gdn_oracle.c`` (plain C, fp64, the definitions of
 Sections 2.2, 4.2 and 5.1 written out).  This module compiles that file with
 gcc on first use and exposes numpy-in / numpy-out wrappers.
+
+Three small definitions are written here in numpy because they move or compare
+values and compute nothing in floating point beyond fp32 additions in a fixed
+order: ``commit_conv`` (convolution state, Section 7), ``tree_mask_to_parent``
+(proposal converter, Section 7) and ``prune_tree`` (confidence-guided pruning,
+Section 6.1).  Pins (tests/test_oracle_pins.py): hand cases and the causal-
+convolution identity for the first, a round trip through independently built
+masks for the second, a hand-worked example plus an independent sort-based
+selection in fp64 on exactly representable scores for the third.  The rule
+switch (``set_rule``) is pinned by the closed form of gated linear attention.
 """
 from __future__ import annotations
 
