@@ -372,6 +372,14 @@ def run_speca(args):
 
     mask_ms = time_util(lambda: speca.tree_mask_to_parent(mask_d, p0["d_offs"], par_out, status))
     prune_ms = time_util(lambda: speca.prune_tree(64, 2.0, 32, p0["d_offs"], p0["d_parent"], logp, oo, op, oi, status))
+    g_sa = torch.Generator(device=dev).manual_seed(1234)
+    sa_q = torch.rand(p0["T"], device=dev, generator=g_sa) * 0.9 + 0.1
+    sa_p = sa_q * (0.5 + torch.rand(p0["T"], device=dev, generator=g_sa))
+    sa_u = torch.rand(p0["T"], device=dev, generator=g_sa)
+    sa_idx = torch.empty(B, 8, dtype=torch.int32, device=dev)
+    sa_len = torch.empty(B, dtype=torch.int32, device=dev)
+    sacc_ms = time_util(lambda: speca.stochastic_accept(B, 8, p0["d_offs"], p0["d_parent"], sa_p, sa_q, sa_u,
+                                                        sa_idx, sa_len, status))
     assert torch.equal(par_out, p0["d_parent"]), "mask converter does not reproduce the parent array"
 
     # --- the same rounds with the commit delayed into the next round's verification ----
@@ -420,7 +428,7 @@ def run_speca(args):
         "gpu_launches": 4 * K,
         "conv_commit": {"ms": conv_ms, "channels": ch, "width": W, "gbs": conv_bytes / (conv_ms * 1e-3) / 1e9,
                         "note": "speca_commit_conv on the accepted paths of one round; outside the timed step"},
-        "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms,
+        "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms, "stochastic_accept_ms": sacc_ms,
                         "note": "one call over the batch's topology (tau = 2, budget 32); integer work outside the timed step"},
         "fused": fused,
         "clocks": clocks,

@@ -161,6 +161,25 @@ int speca_greedy_accept(int32_t batch, int32_t max_depth,
                         int32_t *path_idx, int32_t *path_len, int32_t *next_tok,
                         int32_t *status_word, void *stream);
 
+/* Stochastic posterior selection (the rejection-sampling-style rule of Section 2.1), for callers that
+ * sample instead of decoding greedily.  p_target, p_draft, uniform: float [T], device, packed like the
+ * nodes.  p_draft[t] is the probability the drafter gave node t's token, p_target[t] the probability the
+ * target gives it at t's parent -- for a node with lower-index siblings: in the residual distribution
+ * that remains once those siblings have been rejected, which the caller computes from its logits --
+ * and uniform[t] a number in [0, 1) drawn by the caller.  Node t passes iff
+ * uniform[t] * p_draft[t] < p_target[t] (fp32 product, then comparison; i.e. uniform < min(1, p/q)).
+ * Starting at the committed state the walk moves to the first child, in ascending index, that passes,
+ * and stops when none does; the nodes visited are written to path_idx[b][0..len) (rest -1) and
+ * path_len[b] = len.  For a chain this is the acceptance rule of speculative sampling verbatim.  The
+ * token that follows the accepted path (drawn from the residual at the stopping node, or from the
+ * target distribution if a leaf was reached) needs vocabulary-sized distributions and stays with the
+ * caller.  Integer-exact given the three arrays; bad topology is reported and accepts nothing. */
+int speca_stochastic_accept(int32_t batch, int32_t max_depth,
+                            const int32_t *node_offsets, const int32_t *parent,
+                            const float *p_target, const float *p_draft, const float *uniform,
+                            int32_t *path_idx, int32_t *path_len,
+                            int32_t *status_word, void *stream);
+
 /* Commit (Section 5.1 factor buffering, Eq. 3; Section 5.2 immediate update): gathers
  * the factor records (k, v, alpha, beta) on the accepted path path_idx[b][0..path_len[b])
  * and advances S over them in place, token by token, in fp32.  path_len[b] == 0 leaves

@@ -8,14 +8,17 @@ The arithmetic lives in ``gdn_oracle.c`` (plain C, fp64, the definitions of
 Sections 2.2, 4.2 and 5.1 written out).  This module compiles that file with
 gcc on first use and exposes numpy-in / numpy-out wrappers.
 
-Three small definitions are written here in numpy because they move or compare
+Four small definitions are written here in numpy because they move or compare
 values and compute nothing in floating point beyond fp32 additions in a fixed
 order: ``commit_conv`` (convolution state, Section 7), ``tree_mask_to_parent``
-(proposal converter, Section 7) and ``prune_tree`` (confidence-guided pruning,
-Section 6.1).  Pins (tests/test_oracle_pins.py): hand cases and the causal-
+(proposal converter, Section 7), ``prune_tree`` (confidence-guided pruning,
+Section 6.1) and ``stochastic_accept`` (the rejection-sampling-style rule of
+Section 2.1 as a walk over per-node tests).  Pins (tests/test_oracle_pins.py): hand cases and the causal-
 convolution identity for the first, a round trip through independently built
 masks for the second, a hand-worked example plus an independent sort-based
-selection in fp64 on exactly representable scores for the third.  The rule
+selection in fp64 on exactly representable scores for the third, hand cases, the
+chain's closed-form acceptance-length distribution and an independent
+level-by-level formulation for the fourth.  The rule
 switch (``set_rule``) is pinned by the closed form of gated linear attention.
 """
 from __future__ import annotations
@@ -249,3 +252,34 @@ def prune_tree(node_offsets, parent, logp, tau, budget):
                 out_index.append(i)
         offs.append(len(out_parent))
     return np.asarray(offs, np.int32), np.asarray(out_parent, np.int32), np.asarray(out_index, np.int32)
+
+
+def stochastic_accept(node_offsets, parent, p_target, p_draft, uniform, max_depth: int):
+    """Stochastic posterior selection (the rejection-sampling-style rule of Section 2.1) given per-node
+    probabilities, as the plain walk: from the committed state, look at the children of the current
+    node in ascending index; child t passes iff uniform[t] * p_draft[t] < p_target[t] (fp32 product,
+    i.e. uniform < min(1, p_target / p_draft)); move to the first child that passes; stop when none
+    does (a path longer than max_depth is outside the contract and raises).  Returns (path_idx int32 [B, max_depth] padded with -1,
+    path_len int32 [B])."""
+    node_offsets, parent = _c(node_offsets, np.int32), _c(parent, np.int32)
+    p_target, p_draft, uniform = _c(p_target, np.float32), _c(p_draft, np.float32), _c(uniform, np.float32)
+    B = node_offsets.shape[0] - 1
+    path_idx = np.full((B, int(max_depth)), -1, np.int32)
+    path_len = np.zeros(B, np.int32)
+    for b in range(B):
+        base, n = int(node_offsets[b]), int(node_offsets[b + 1] - node_offsets[b])
+        cur, d = -1, 0
+        while True:
+            nxt = -1
+            for t in range(cur + 1, n):
+                if parent[base + t] == cur and np.float32(uniform[base + t] * p_draft[base + t]) < p_target[base + t]:
+                    nxt = t
+                    break
+            if nxt < 0:
+                break
+            if d == max_depth:
+                raise ValueError("accepted path longer than max_depth")
+            path_idx[b, d] = nxt
+            cur, d = nxt, d + 1
+        path_len[b] = d
+    return path_idx, path_len

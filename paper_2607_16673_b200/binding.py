@@ -27,7 +27,7 @@ RULE_GATED_DELTA, RULE_GATED_NO_ERASE = 0, 1
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
            "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv",
-           "speca_tree_mask_to_parent", "speca_prune_tree"]
+           "speca_tree_mask_to_parent", "speca_prune_tree", "speca_stochastic_accept"]
 NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.speca_tree_mask_to_parent.restype = ctypes.c_int
         L.speca_prune_tree.argtypes = [i32, i32, ctypes.c_float, i32] + [vp] * 8
         L.speca_prune_tree.restype = ctypes.c_int
+        L.speca_stochastic_accept.argtypes = [i32, i32] + [vp] * 9
+        L.speca_stochastic_accept.restype = ctypes.c_int
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
                      "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"):
             getattr(L, name).restype = ctypes.c_int
@@ -197,6 +199,20 @@ def greedy_accept(batch: int, max_depth: int, node_offsets, parent, draft_tok, t
         _ptr(path_idx, i32, (batch, max_depth), "path_idx"), _ptr(path_len, i32, (batch,), "path_len"),
         _ptr(next_tok, i32, (batch,), "next_tok"), _ptr(status, i32, (1,), "status"), _stream())
     _check(rc, "speca_greedy_accept")
+
+
+def stochastic_accept(batch: int, max_depth: int, node_offsets, parent, p_target, p_draft, uniform,
+                      path_idx, path_len, status) -> None:
+    """speca_stochastic_accept: the walk over first passing children (uniform * p_draft < p_target)."""
+    i32, f32 = torch.int32, torch.float32
+    shape = tuple(parent.shape)
+    rc = lib().speca_stochastic_accept(
+        int(batch), int(max_depth), _ptr(node_offsets, i32, (batch + 1,), "node_offsets"),
+        _ptr(parent, i32, None, "parent"), _ptr(p_target, f32, shape, "p_target"),
+        _ptr(p_draft, f32, shape, "p_draft"), _ptr(uniform, f32, shape, "uniform"),
+        _ptr(path_idx, i32, (batch, max_depth), "path_idx"), _ptr(path_len, i32, (batch,), "path_len"),
+        _ptr(status, i32, (1,), "status"), _stream())
+    _check(rc, "speca_stochastic_accept")
 
 
 def commit(dims: Dims, S, k, v, alpha, beta, node_offsets, total_nodes, parent, path_idx, path_len, status) -> None:

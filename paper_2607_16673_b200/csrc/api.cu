@@ -202,6 +202,18 @@ int speca_greedy_accept(int32_t batch, int32_t max_depth, const int32_t *node_of
                                  static_cast<cudaStream_t>(stream)));
 }
 
+int speca_stochastic_accept(int32_t batch, int32_t max_depth, const int32_t *node_offsets,
+                            const int32_t *parent, const float *p_target, const float *p_draft,
+                            const float *uniform, int32_t *path_idx, int32_t *path_len,
+                            int32_t *status_word, void *stream)
+{
+    if (!node_offsets || !parent || !p_target || !p_draft || !uniform || !path_idx || !path_len || !status_word)
+        return SPECA_ERR_NULL;
+    if (batch < 1 || max_depth < 1 || max_depth > 16) return SPECA_ERR_RANGE;
+    return cuda_rc(launch_stochastic_accept(batch, max_depth, node_offsets, parent, p_target, p_draft, uniform,
+                                            path_idx, path_len, status_word, static_cast<cudaStream_t>(stream)));
+}
+
 int speca_commit(const speca_dims *dims, float *S, const uint16_t *k, const uint16_t *v,
                  const float *alpha, const float *beta, const int32_t *node_offsets, int32_t total_nodes,
                  const int32_t *parent_or_null, const int32_t *path_idx, const int32_t *path_len,

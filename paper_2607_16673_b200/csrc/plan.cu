@@ -194,6 +194,63 @@ accept_kernel(int32_t B, int32_t max_depth, const int32_t *__restrict__ node_off
     }
 }
 
+// Stochastic posterior selection given per-node probabilities: one warp per sequence.
+// Node t passes its own test iff uniform[t] * p_draft[t] < p_target[t] (uniform < min(1, p/q),
+// written without the division; one fp32 product and one comparison).  From the committed state
+// the walk takes, among the children of the current node in ascending index, the first that
+// passes, and stops when none does.  A node is therefore on the accepted path iff it and all
+// its ancestors are "chosen": passing, with no passing sibling of lower index.
+__global__ void __launch_bounds__(128)
+stochastic_accept_kernel(int32_t B, int32_t max_depth, const int32_t *__restrict__ node_offsets,
+                         const int32_t *__restrict__ parent, const float *__restrict__ p_target,
+                         const float *__restrict__ p_draft, const float *__restrict__ uniform,
+                         int32_t *__restrict__ path_idx, int32_t *__restrict__ path_len, int32_t *status)
+{
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const int base = node_offsets[b];
+    const int n = node_offsets[b + 1] - base;
+    int fault = 0;
+    if (base < 0 || n < 0) fault = SPECA_STATUS_BAD_OFFSETS;
+    if (n > 0x10000) fault |= SPECA_STATUS_TOO_MANY;
+    auto passes = [&](int t) { return __fmul_rn(uniform[base + t], p_draft[base + t]) < p_target[base + t]; };
+    int best = -1;                     // (depth << 16) | (0xffff - index) of the deepest node whose root path is all chosen
+    if (!fault) {
+        for (int t = lane; t < n; t += 32) {
+            int d = 0, ok = 1;
+            for (int a = t; a >= 0;) {
+                const int pa = parent[base + a];
+                if (pa < -1 || pa >= a) { fault |= SPECA_STATUS_BAD_PARENT; ok = 0; break; }
+                if (!passes(a)) { ok = 0; break; }
+                // a lower-index sibling that passes is taken instead
+                for (int s2 = pa + 1; s2 < a; ++s2)
+                    if (parent[base + s2] == pa && passes(s2)) { ok = 0; break; }
+                if (!ok) break;
+                if (++d > max_depth) { fault |= SPECA_STATUS_TOO_DEEP; ok = 0; break; }
+                a = pa;
+            }
+            if (ok) best = max(best, (d << 16) | (0xffff - t));
+        }
+    }
+    for (int off = 16; off; off >>= 1) {
+        best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+        fault |= __shfl_xor_sync(0xffffffffu, fault, off);
+    }
+    if (lane != 0) return;
+    if (fault) {                       // skip the sequence: nothing accepted
+        atomicOr(status, fault);
+        best = -1;
+    }
+    const int len = best < 0 ? 0 : (best >> 16);
+    int node = best < 0 ? -1 : 0xffff - (best & 0xffff);
+    path_len[b] = len;
+    for (int d = max_depth - 1; d >= 0; --d) {
+        if (d < len) { path_idx[b * max_depth + d] = node; node = parent[base + node]; }
+        else path_idx[b * max_depth + d] = -1;
+    }
+}
+
 // Pending accepted paths of the fused commit-and-verify call, one thread per sequence:
 // the same checks the stand-alone commit makes (length, node range, parent chain when the
 // parent array is given), plus a node count within max_nodes.  A bad path is reported and
@@ -462,6 +519,16 @@ int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, con
     accept_kernel<<<(B + warps - 1) / warps, warps * 32, 0, st>>>(
         B, max_depth, node_offsets, parent, draft_tok, target_tok, root_target_tok, path_idx, path_len,
         next_tok, status);
+    return int(cudaGetLastError());
+}
+
+int launch_stochastic_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
+                             const float *p_target, const float *p_draft, const float *uniform,
+                             int32_t *path_idx, int32_t *path_len, int32_t *status, cudaStream_t st)
+{
+    const int warps = 4;
+    stochastic_accept_kernel<<<(B + warps - 1) / warps, warps * 32, 0, st>>>(
+        B, max_depth, node_offsets, parent, p_target, p_draft, uniform, path_idx, path_len, status);
     return int(cudaGetLastError());
 }
 

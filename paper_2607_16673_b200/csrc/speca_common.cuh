@@ -114,6 +114,9 @@ int launch_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, con
                   const int32_t *draft_tok, const int32_t *target_tok, const int32_t *root_target_tok,
                   int32_t *path_idx, int32_t *path_len, int32_t *next_tok, int32_t *status,
                   cudaStream_t st);
+int launch_stochastic_accept(int32_t B, int32_t max_depth, const int32_t *node_offsets, const int32_t *parent,
+                             const float *p_target, const float *p_draft, const float *uniform,
+                             int32_t *path_idx, int32_t *path_len, int32_t *status, cudaStream_t st);
 
 // Number of on-chip state slots the light-children-first walk can need for a tree of
 // at most n nodes: a node saves its state only if it has two children with

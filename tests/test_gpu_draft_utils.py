@@ -78,3 +78,56 @@ def test_prune_tree(tau, budget):
     assert np.array_equal(op.cpu().numpy()[:n], rp) and np.array_equal(oi.cpu().numpy()[:n], ri)
     # the pruned topology is a valid input of the verification path
     assert np.all(rp < np.arange(n) - ro[np.searchsorted(ro, np.arange(n), side="right") - 1]) or n == 0
+
+
+def test_stochastic_accept_matches_the_walk():
+    """speca_stochastic_accept against the oracle's walk: paths and lengths bit-exact, over many batches."""
+    rng = np.random.default_rng(63)
+    for trial in range(6):
+        parents, offs = batch(rng, 48, 1, 64)
+        if trial == 0:
+            parents[1] = synth.chain_parent(8)
+            parents[2] = synth.chain_parent(1)
+            offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+        parent = np.concatenate(parents).astype(np.int32)
+        T = int(offs[-1])
+        p_draft = rng.uniform(0.02, 1.0, T).astype(np.float32)
+        # ratios p/q spread around 1 so that paths of every length occur; some exact ties u * q == p
+        p_target = (p_draft * rng.choice([0.25, 0.5, 1.0, 2.0], T)).astype(np.float32)
+        uniform = rng.random(T, dtype=np.float32)
+        ties = rng.random(T) < 0.05
+        uniform[ties] = (p_target[ties] / p_draft[ties]).astype(np.float32)
+        uniform = np.minimum(uniform, np.float32(0.99999994))
+        B = len(parents)
+        pidx = torch.full((B, 8), -9, dtype=torch.int32, device="cuda")
+        plen = torch.full((B,), -9, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        speca.stochastic_accept(B, 8, t(offs), t(parent), t(p_target), t(p_draft), t(uniform), pidx, plen, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        pi, pl = oracle.stochastic_accept(offs, parent, p_target, p_draft, uniform, 8)
+        assert np.array_equal(plen.cpu().numpy(), pl)
+        assert np.array_equal(pidx.cpu().numpy(), pi)
+        assert pl.max() >= 3 and (pl == 0).any()
+
+
+def test_stochastic_accept_reports_bad_topology_and_accepts_nothing_there():
+    parents = [synth.chain_parent(4), np.array([-1, 1, 0], np.int32), synth.chain_parent(3)]
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    parent = np.concatenate(parents).astype(np.int32)
+    T = int(offs[-1])
+    one = torch.ones(T, device="cuda")
+    zero = torch.zeros(T, device="cuda")
+    pidx = torch.full((3, 8), -9, dtype=torch.int32, device="cuda")
+    plen = torch.full((3,), -9, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    speca.stochastic_accept(3, 8, t(offs), t(parent), one, one, zero, pidx, plen, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & speca.STATUS_BAD_PARENT
+    assert plen.cpu().tolist() == [4, 0, 3]
+    assert pidx.cpu()[0].tolist() == [0, 1, 2, 3, -1, -1, -1, -1] and pidx.cpu()[1].tolist() == [-1] * 8
+    # a chain longer than max_depth is reported, not truncated
+    status.zero_()
+    speca.stochastic_accept(3, 3, t(offs), t(parent), one, one, zero, pidx[:, :3].contiguous(), plen, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & speca.STATUS_TOO_DEEP and plen.cpu().tolist()[0] == 0

@@ -8,7 +8,8 @@ routes that share nothing with oracle/gdn_oracle.c.
   * structural invariants: chain == repeated decode, single-path tree == chain,
     commit == sequential recurrence, sibling isolation, linearity in (S0, V),
     row independence, relabelling by another topological order
-  * acceptance: brute force over all root paths, hand cases
+  * acceptance: brute force over all root paths, hand cases; the stochastic rule: hand cases, min(1, p/q),
+    the closed-form length distribution on chains, a level-free restatement
   * byte counts printed by the paper (state, snapshots, factor buffer)
 """
 import itertools
@@ -555,6 +556,69 @@ def test_pruning_hand_case_and_selection_properties():
             newpar = pp[oo[b]:oo[b + 1]]
             for r, i in enumerate(got):                # ancestor-closed and re-indexed consistently
                 assert (par[i] < 0 and newpar[r] == -1) or got[newpar[r]] == par[i]
+
+
+def test_stochastic_accept_hand_cases_closed_form_and_level_formulation():
+    """The rejection-sampling-style rule of Section 2.1 as a walk over per-node tests."""
+    acc = lambda par, pt, pd, u, md=8: [x.tolist() for x in oracle.stochastic_accept(
+        np.array([0, len(par)], np.int32), np.asarray(par, np.int32), np.asarray(pt, np.float32),
+        np.asarray(pd, np.float32), np.asarray(u, np.float32), md)]
+    # chain of 4, ratios p/q = 0.5, 2, 0.25, 1: accepted while u < min(1, p/q)
+    par, pt, pd = [-1, 0, 1, 2], [0.25, 0.5, 0.125, 0.5], [0.5, 0.25, 0.5, 0.5]
+    assert acc(par, pt, pd, [0.49, 0.99, 0.24, 0.99]) == [[[0, 1, 2, 3, -1, -1, -1, -1]], [4]]
+    assert acc(par, pt, pd, [0.49, 0.99, 0.25, 0.0])[1] == [2]          # u == ratio is a rejection (strict <)
+    assert acc(par, pt, pd, [0.5, 0.0, 0.0, 0.0])[1] == [0]             # the first test already fails
+    assert acc(par, [0, 0, 0, 0], pd, [0, 0, 0, 0])[1] == [0]           # target probability 0 never passes
+    # tree: 0 -> {1, 2}, 2 -> {3}; the first passing child in index order is taken, later siblings are not looked at
+    par, one = [-1, 0, 0, 2], [1.0] * 4
+    assert acc(par, [1, 0.1, 1, 1], one, [0.5, 0.5, 0.5, 0.5]) == [[[0, 2, 3, -1, -1, -1, -1, -1]], [3]]
+    assert acc(par, [1, 0.9, 1, 1], one, [0.5, 0.5, 0.5, 0.5]) == [[[0, 1, -1, -1, -1, -1, -1, -1]], [2]]
+    assert acc(par, [1, 0.1, 0.1, 1], one, [0.5, 0.5, 0.5, 0.0])[1] == [1]   # node 3 passes but is never reached
+    with pytest.raises(ValueError):
+        acc([-1, 0, 1], [1, 1, 1], [1, 1, 1], [0, 0, 0], md=2)
+    # the acceptance probability of one node is min(1, p/q): sweep u over a grid
+    for ptv, pdv in [(0.3, 0.6), (0.6, 0.3), (0.125, 1.0), (0.5, 0.5)]:
+        grid = (np.arange(4096) / 4096.0).astype(np.float32)
+        n_acc = sum(acc([-1], [ptv], [pdv], [uu])[1][0] for uu in grid[::16])
+        assert abs(n_acc / 256.0 - min(1.0, ptv / pdv)) <= 1.0 / 256
+    # with it the one-step output distribution equals the target's (speculative sampling's defining property):
+    # P(out = x) = q(x) a(x) + (1 - sum_y q(y) a(y)) r(x), a = min(1, p/q), r = normalised max(0, p - q)
+    p3, q3 = np.array([0.5, 0.3, 0.2]), np.array([0.2, 0.3, 0.5])
+    a3 = np.minimum(1.0, p3 / q3)
+    r3 = np.maximum(0.0, p3 - q3)
+    np.testing.assert_allclose(q3 * a3 + (1 - (q3 * a3).sum()) * r3 / r3.sum(), p3, atol=1e-15)
+    # closed form on chains: p = a q at every node -> P(len >= k) = a^k, so E[len] = a (1 - a^n) / (1 - a)
+    rng = np.random.default_rng(77)
+    B, n, a = 20000, 6, 0.7
+    offs = (np.arange(B + 1) * n).astype(np.int32)
+    parent = np.tile(np.arange(-1, n - 1, dtype=np.int32), B)
+    pd_ = rng.uniform(0.05, 1.0, B * n).astype(np.float32)
+    pt_ = (np.float32(a) * pd_).astype(np.float32)
+    _, ln = oracle.stochastic_accept(offs, parent, pt_, pd_, rng.random(B * n, dtype=np.float32), 8)
+    mean = a * (1 - a ** n) / (1 - a)
+    assert abs(ln.mean() - mean) < 4 * 1.6 / np.sqrt(B)                     # std of the length is below 1.6
+    assert abs((ln == n).mean() - a ** n) < 4 * np.sqrt(a ** n * (1 - a ** n) / B)
+    # an independent formulation: a node is on the path iff it and all its ancestors pass and have no passing
+    # sibling of lower index; resolved for all nodes at once from the parent array
+    parents = [synth.random_tree_parent(int(rng.integers(1, 48)), 8, 4, rng) for _ in range(64)]
+    offs = np.concatenate([[0], np.cumsum([len(pp) for pp in parents])]).astype(np.int32)
+    parent = np.concatenate(parents).astype(np.int32)
+    T = int(offs[-1])
+    pd_ = rng.uniform(0.05, 1.0, T).astype(np.float32)
+    pt_ = rng.uniform(0.0, 1.0, T).astype(np.float32)
+    u_ = rng.random(T, dtype=np.float32)
+    pi, pl = oracle.stochastic_accept(offs, parent, pt_, pd_, u_, 8)
+    passes = (u_ * pd_) < pt_
+    for b, par in enumerate(parents):
+        ps = passes[offs[b]:offs[b + 1]]
+        first = {}                                       # parent -> lowest passing child
+        for t in range(len(par)):
+            if ps[t]:
+                first.setdefault(int(par[t]), t)
+        on = [t for t in range(len(par))
+              if all(first.get(int(par[x])) == x for x in synth.root_path(par, t))]
+        on.sort(key=lambda t: len(synth.root_path(par, t)))
+        assert pi[b, :pl[b]].tolist() == on and pl[b] == len(on)
 
 
 def test_rule_without_erase_is_gated_linear_attention():
