@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the speculative verify -> accept -> commit path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4|paper256|trees64|chains8|paper] [--impl reference]
 
 One "step" is one round of the whole hot path over one batch of synthetic draft input:
 plan + verify (all layers, heads, nodes) -> greedy accept -> commit, with the committed
@@ -38,6 +38,9 @@ WORKLOADS = {
                                     "64 seq with 64-node trees (depth<=8)"),
     "cfg4": (24, 32, 16, 128, 256, "32 seq x 24 layers x 16 heads, d_k=128 d_v=256; ragged trees of 8..64 nodes (depth<=8)"),
     # the paper's target shape (h_v = 8, d_k = d_v = 256, 24 layers) served in a batch
+    # the two unit types of cfg5 on their own (same shape): what a unit of each kind costs
+    "trees64": (24, 128, 16, 128, 256, "128 seq x 24 layers x 16 heads, d_k=128 d_v=256; every sequence a 64-node tree (depth<=8)"),
+    "chains8": (24, 128, 16, 128, 256, "128 seq x 24 layers x 16 heads, d_k=128 d_v=256; every sequence an 8-token chain"),
     "paper256": (24, 64, 8, 256, 256, "64 seq x 24 layers x 8 heads, d_k=d_v=256 (the paper's target shape); 32 seq with "
                                       "8-token chains + 32 seq with top-4 proposal trees of 16..32 nodes (depth 4..8)"),
 }
@@ -50,7 +53,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS) + ["paper"],
-                    help="cfg5 (default), cfg4, or 'paper': the paper's own target shape and proposal shapes (Table 1)")
+                    help="cfg5 (default), cfg4, paper256, trees64 / chains8 (cfg5's unit types on their own), or 'paper': "
+                         "the paper's own target shape and proposal shapes (Table 1)")
     ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
     ap.add_argument("--route", type=int, default=0, help="0 auto, 1 serial, 2 factorized")
     ap.add_argument("--e2e-steps", type=int, default=6)
@@ -65,18 +69,27 @@ def parse_args():
 # ---------------------------------------------------------------------------
 # workload description (host side: topology and token ids; no method arithmetic)
 # ---------------------------------------------------------------------------
+def workload_parents(name: str, rng, n: int):
+    """Parent arrays of n sequences of a workload."""
+    from paper_2607_16673_b200 import synth
+    if name == "cfg5":
+        return synth.mixed_chain_tree_batch(rng, n, 8, 64, 8)
+    if name == "trees64":
+        return [synth.random_tree_parent(64, 8, 4, rng) for _ in range(n)]
+    if name == "chains8":
+        return [synth.chain_parent(8) for _ in range(n)]
+    if name == "paper256":
+        return ([synth.chain_parent(8) for _ in range(n // 2)] +
+                [synth.proposal_tree_parent(4, int(rng.integers(4, 9)), int(rng.integers(16, 33)), rng, 8)
+                 for _ in range(n - n // 2)])
+    return synth.ragged_tree_batch(rng, n, 8, 64, 8)
+
+
 def host_round_inputs(name: str, B: int, seed: int):
     """Topology and token ids of one round, on the host."""
     from paper_2607_16673_b200 import synth
     rng = np.random.default_rng(seed)
-    if name == "cfg5":
-        parents = synth.mixed_chain_tree_batch(rng, B, 8, 64, 8)
-    elif name == "paper256":
-        parents = [synth.chain_parent(8) for _ in range(B // 2)]
-        parents += [synth.proposal_tree_parent(4, int(rng.integers(4, 9)), int(rng.integers(16, 33)), rng, 8)
-                    for _ in range(B - B // 2)]
-    else:
-        parents = synth.ragged_tree_batch(rng, B, 8, 64, 8)
+    parents = workload_parents(name, rng, B)
     sizes = [len(p) for p in parents]
     offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
     parent = np.concatenate(parents).astype(np.int32)
@@ -591,14 +604,7 @@ def oracle_sample_problem(workload: str, H: int, dk: int, dv: int, n_units: int,
     trees for cfg5 (ragged trees for cfg4), repacked as independent single-head sequences."""
     from paper_2607_16673_b200 import synth
     rng = np.random.default_rng(seed)
-    if workload == "cfg5":
-        parents = synth.mixed_chain_tree_batch(rng, n_units, 8, 64, 8)
-    elif workload == "paper256":
-        parents = [synth.chain_parent(8) for _ in range(n_units // 2)]
-        parents += [synth.proposal_tree_parent(4, int(rng.integers(4, 9)), int(rng.integers(16, 33)), rng, 8)
-                    for _ in range(n_units - n_units // 2)]
-    else:
-        parents = synth.ragged_tree_batch(rng, n_units, 8, 64, 8)
+    parents = workload_parents(workload, rng, n_units)
     return synth.make_problem(seed, 1, 1, dk, dv, parents)
 
 
