@@ -476,6 +476,68 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
     }
 }
 
+// packed fp32 pairs (sm_100: two IEEE operations per instruction)
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// The 8-level step with the levels taken two at a time by packed fp32 FMAs (each half an IEEE
+// fma): the pairs (cU[2i], cU[2i+1]) come out of the 128-bit loads as they are, and the stack is
+// read as the matching pairs of levels.  Level 7 is never an ancestor (a node has at most 7), so
+// its slot carries v through the u step, paired with cV, and the node's own u afterwards if the
+// node is at depth 8; cO[7] is zero otherwise.  Used by the plain kernel (it is no gain in the
+// fused one, whose update role competes for the same issue slots).
+template <int TP>
+__device__ __forceinline__ void node_step_packed(float (&ustk)[TP][kMaxDepth], const float *cf, const float (&Rv)[TP],
+                                                 const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
+                                                 float (&o_out)[TP], int &off)
+{
+    const ulonglong2 a0 = *reinterpret_cast<const ulonglong2 *>(cf + 0), a1 = *reinterpret_cast<const ulonglong2 *>(cf + 4);
+    const ulonglong2 b0 = *reinterpret_cast<const ulonglong2 *>(cf + 8), b1 = *reinterpret_cast<const ulonglong2 *>(cf + 12);
+    const float4 s = *reinterpret_cast<const float4 *>(cf + 16);
+    const int d1 = __float_as_int(s.z);
+    off = __float_as_int(s.w);
+#pragma unroll
+    for (int t = 0; t < TP; ++t) {
+        ustk[t][7] = vv[t];
+        unsigned long long acc = mul2(a0.x, pack2(ustk[t][0], ustk[t][1]));
+        acc = fma2(a0.y, pack2(ustk[t][2], ustk[t][3]), acc);
+        acc = fma2(a1.x, pack2(ustk[t][4], ustk[t][5]), acc);
+        acc = fma2(a1.y, pack2(ustk[t][6], ustk[t][7]), acc);
+        float e, f;
+        unpack2(acc, e, f);
+        const float u = fmaf(s.x, Rv[t], e + f);
+#pragma unroll
+        for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        acc = mul2(b0.x, pack2(ustk[t][0], ustk[t][1]));
+        acc = fma2(b0.y, pack2(ustk[t][2], ustk[t][3]), acc);
+        acc = fma2(b1.x, pack2(ustk[t][4], ustk[t][5]), acc);
+        acc = fma2(b1.y, pack2(ustk[t][6], ustk[t][7]), acc);
+        unpack2(acc, e, f);
+        o_out[t] = fmaf(s.y, Gv[t], e + f);
+        u_out[t] = u;
+    }
+}
+
 // The same step for trees up to MAXD levels deep (the coefficient record is cU[MAXD-1] cV cO[MAXD] cR cG
 // depth-1 offset).  Used for MAXD = 16; the 8-level form above is kept as it is because the shape of its
 // two accumulation chains was tuned.
@@ -1138,7 +1200,8 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                         v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
                     }
                     if constexpr (DEEP) node_step_deep<TP, MAXD>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
-                    else node_step<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
+                    else if constexpr (FUSED) node_step<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
+                    else node_step_packed<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
                     if (p0 + i < n) {
                         if (TP == 2) {
                             *reinterpret_cast<float2 *>(o_row + off) = make_float2(oo[0], oo[TP - 1]);
