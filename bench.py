@@ -393,6 +393,9 @@ def run_speca(args):
     sa_len = torch.empty(B, dtype=torch.int32, device=dev)
     sacc_ms = time_util(lambda: speca.stochastic_accept(B, 8, p0["d_offs"], p0["d_parent"], sa_p, sa_q, sa_u,
                                                         sa_idx, sa_len, status))
+    ch_head = torch.empty(p0["T"], dtype=torch.int32, device=dev)
+    ch_cnt = torch.empty(B, dtype=torch.int32, device=dev)
+    chain_ms = time_util(lambda: speca.chain_decompose(64, p0["d_offs"], p0["d_parent"], ch_head, ch_cnt, status))
     assert torch.equal(par_out, p0["d_parent"]), "mask converter does not reproduce the parent array"
 
     # --- the same rounds with the commit delayed into the next round's verification ----
@@ -441,7 +444,7 @@ def run_speca(args):
         "gpu_launches": 4 * K,
         "conv_commit": {"ms": conv_ms, "channels": ch, "width": W, "gbs": conv_bytes / (conv_ms * 1e-3) / 1e9,
                         "note": "speca_commit_conv on the accepted paths of one round; outside the timed step"},
-        "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms, "stochastic_accept_ms": sacc_ms,
+        "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms, "stochastic_accept_ms": sacc_ms, "chain_decompose_ms": chain_ms,
                         "note": "one call over the batch's topology (tau = 2, budget 32); integer work outside the timed step"},
         "fused": fused,
         "clocks": clocks,

@@ -252,10 +252,23 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S,
  * nodes whose parent is kept -- with log-probabilities (<= 0) q never increases along a path and the last
  * rule changes nothing.  The kept nodes of all sequences are written packed, in their original order:
  * out_offsets [B+1], out_parent [.] (re-indexed, local), out_index [.] (original local index); out_parent
- * and out_index need room for T entries.  A sequence with bad topology is reported and contributes nothing. */
+ * and out_index need room for T entries.  A sequence with bad topology is reported and contributes nothing.
+ *
+ * speca_chain_decompose: the heavy-light chain decomposition of Section 4.3 (the scheduling unit of the
+ * paper's hybrid route: node-disjoint chains that together cover the tree, each verifiable as a chain from
+ * the boundary state of the node it hangs off).  The heavy child of a node is its child with the largest
+ * subtree (lowest index on ties); a node continues its parent's chain iff it is that heavy child, every
+ * other node -- and every child of the committed state -- heads a chain.  Writes chain_head[node_offsets[b]
+ * + i] = local index of the first node of i's chain and n_chains[b] = the number of chains.  On any root
+ * path at most floor(log2(n)) chains are entered below the first.  A sequence with bad topology is
+ * reported, gets n_chains[b] = 0 and its chain_head entries are left untouched. */
 int speca_tree_mask_to_parent(int32_t batch, int32_t max_nodes, const uint8_t *mask,
                               const int32_t *node_offsets, int32_t *parent,
                               int32_t *status_word, void *stream);
+int speca_chain_decompose(int32_t batch, int32_t max_nodes,
+                          const int32_t *node_offsets, const int32_t *parent,
+                          int32_t *chain_head, int32_t *n_chains,
+                          int32_t *status_word, void *stream);
 int speca_prune_tree(int32_t batch, int32_t max_nodes, float tau, int32_t budget,
                      const int32_t *node_offsets, const int32_t *parent, const float *logp,
                      int32_t *out_offsets, int32_t *out_parent, int32_t *out_index,

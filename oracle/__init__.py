@@ -8,17 +8,20 @@ The arithmetic lives in ``gdn_oracle.c`` (plain C, fp64, the definitions of
 Sections 2.2, 4.2 and 5.1 written out).  This module compiles that file with
 gcc on first use and exposes numpy-in / numpy-out wrappers.
 
-Four small definitions are written here in numpy because they move or compare
+Five small definitions are written here in numpy because they move or compare
 values and compute nothing in floating point beyond fp32 additions in a fixed
 order: ``commit_conv`` (convolution state, Section 7), ``tree_mask_to_parent``
 (proposal converter, Section 7), ``prune_tree`` (confidence-guided pruning,
-Section 6.1) and ``stochastic_accept`` (the rejection-sampling-style rule of
-Section 2.1 as a walk over per-node tests).  Pins (tests/test_oracle_pins.py): hand cases and the causal-
+Section 6.1), ``stochastic_accept`` (the rejection-sampling-style rule of
+Section 2.1 as a walk over per-node tests) and ``chain_decompose`` (the
+heavy-light chains of Section 4.3).  Pins (tests/test_oracle_pins.py): hand cases and the causal-
 convolution identity for the first, a round trip through independently built
 masks for the second, a hand-worked example plus an independent sort-based
 selection in fp64 on exactly representable scores for the third, hand cases, the
 chain's closed-form acceptance-length distribution and an independent
-level-by-level formulation for the fourth.  The rule
+level-by-level formulation for the fourth, the chains the paper prints for its
+example (Section 4.3), the partition and path properties and the logarithmic
+bound on chain changes along a root path for the fifth.  The rule
 switch (``set_rule``) is pinned by the closed form of gated linear attention.
 """
 from __future__ import annotations
@@ -283,3 +286,32 @@ def stochastic_accept(node_offsets, parent, p_target, p_draft, uniform, max_dept
             cur, d = nxt, d + 1
         path_len[b] = d
     return path_idx, path_len
+
+
+def chain_decompose(node_offsets, parent):
+    """Heavy-light chain decomposition (Section 4.3), written out: subtree sizes by a pass from the last
+    node to the first, the heavy child of a node = its child with the largest subtree (lowest index on
+    ties), and chains grown from their heads: a node continues its parent's chain iff it is the heavy
+    child; children of the committed state head chains.  Returns (chain_head int32 [T], n_chains int32
+    [B]): for every node the local index of the first node of its chain."""
+    node_offsets, parent = _c(node_offsets, np.int32), _c(parent, np.int32)
+    B = node_offsets.shape[0] - 1
+    chain_head = np.zeros(parent.shape[0], np.int32)
+    n_chains = np.zeros(B, np.int32)
+    for b in range(B):
+        base, n = int(node_offsets[b]), int(node_offsets[b + 1] - node_offsets[b])
+        par = parent[base:base + n]
+        size = [1] * n
+        for t in range(n - 1, -1, -1):
+            if par[t] >= 0:
+                size[par[t]] += size[t]
+        heavy = [-1] * n
+        for t in range(n):                               # ascending: the first child of maximal size wins
+            p = par[t]
+            if p >= 0 and (heavy[p] < 0 or size[t] > size[heavy[p]]):
+                heavy[p] = t
+        for t in range(n):                               # parents come before children
+            p = par[t]
+            chain_head[base + t] = chain_head[base + p] if (p >= 0 and heavy[p] == t) else t
+            n_chains[b] += int(chain_head[base + t] == t)
+    return chain_head, n_chains

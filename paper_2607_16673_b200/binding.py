@@ -27,7 +27,8 @@ RULE_GATED_DELTA, RULE_GATED_NO_ERASE = 0, 1
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",
            "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept", "speca_commit",
            "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv",
-           "speca_tree_mask_to_parent", "speca_prune_tree", "speca_stochastic_accept"]
+           "speca_tree_mask_to_parent", "speca_prune_tree", "speca_stochastic_accept",
+           "speca_chain_decompose"]
 NOALLOC_MAX_BATCH, NOALLOC_MAX_NODES = 256, 16384
 
 
@@ -92,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.speca_prune_tree.argtypes = [i32, i32, ctypes.c_float, i32] + [vp] * 8
         L.speca_prune_tree.restype = ctypes.c_int
         L.speca_stochastic_accept.argtypes = [i32, i32] + [vp] * 9
+        L.speca_chain_decompose.argtypes = [i32, i32] + [vp] * 6
+        L.speca_chain_decompose.restype = ctypes.c_int
         L.speca_stochastic_accept.restype = ctypes.c_int
         for name in ("speca_decode_step", "speca_verify_chain", "speca_verify_tree", "speca_greedy_accept",
                      "speca_commit", "speca_verify_tree_noalloc", "speca_commit_verify_tree", "speca_commit_conv"):
@@ -301,3 +304,14 @@ def prune_tree(max_nodes: int, tau: float, budget: int, node_offsets, parent, lo
                                 _ptr(out_parent, i32, (T,), "out_parent"), _ptr(out_index, i32, (T,), "out_index"),
                                 _ptr(status, i32, (1,), "status"), _stream())
     _check(rc, "speca_prune_tree")
+
+
+def chain_decompose(max_nodes: int, node_offsets, parent, chain_head, n_chains, status) -> None:
+    """speca_chain_decompose: heavy-light chains; chain_head[t] = first node of t's chain, n_chains per sequence."""
+    i32 = torch.int32
+    B = node_offsets.numel() - 1
+    T = parent.numel()
+    rc = lib().speca_chain_decompose(int(B), int(max_nodes), _ptr(node_offsets, i32, (B + 1,), "node_offsets"),
+                                     _ptr(parent, i32, (T,), "parent"), _ptr(chain_head, i32, (T,), "chain_head"),
+                                     _ptr(n_chains, i32, (B,), "n_chains"), _ptr(status, i32, (1,), "status"), _stream())
+    _check(rc, "speca_chain_decompose")

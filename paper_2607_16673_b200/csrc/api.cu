@@ -257,6 +257,15 @@ int speca_prune_tree(int32_t batch, int32_t max_nodes, float tau, int32_t budget
                                 out_index, status_word, static_cast<cudaStream_t>(stream)));
 }
 
+int speca_chain_decompose(int32_t batch, int32_t max_nodes, const int32_t *node_offsets, const int32_t *parent,
+                          int32_t *chain_head, int32_t *n_chains, int32_t *status_word, void *stream)
+{
+    if (!node_offsets || !parent || !chain_head || !n_chains || !status_word) return SPECA_ERR_NULL;
+    if (batch < 1 || max_nodes < 1 || max_nodes > 1024) return SPECA_ERR_RANGE;
+    return cuda_rc(launch_chain_decompose(batch, max_nodes, node_offsets, parent, chain_head, n_chains, status_word,
+                                          static_cast<cudaStream_t>(stream)));
+}
+
 int speca_commit_conv(int32_t n_layers, int32_t batch, int32_t channels, int32_t width, int32_t max_depth,
                       uint16_t *C, const uint16_t *x, const int32_t *node_offsets, int32_t total_nodes,
                       const int32_t *path_idx, const int32_t *path_len, int32_t *status_word, void *stream)

@@ -374,6 +374,61 @@ mask_to_parent_kernel(int32_t N, const uint8_t *__restrict__ mask, const int32_t
     for (int i = threadIdx.x; i < n; i += blockDim.x) parent[base + i] = sm[N + i];
 }
 
+// Heavy-light chain decomposition (Section 4.3): one CTA per sequence, thread i owns node i.  The heavy
+// child of a node is its child with the largest subtree (lowest index on ties); a node continues its
+// parent's chain iff it is that heavy child, otherwise it heads a chain of its own (so does every child
+// of the committed state).  Subtree sizes are integer sums over ancestor walks, the heavy child an
+// integer maximum: both are exact whatever the order of the atomics.
+__global__ void __launch_bounds__(256)
+chain_decompose_kernel(int32_t N, const int32_t *__restrict__ node_offsets, const int32_t *__restrict__ parent,
+                       int32_t *__restrict__ chain_head, int32_t *__restrict__ n_chains, int32_t *status)
+{
+    extern __shared__ int32_t sm[];                     // [N] subtree size, [N] key of the heavy child
+    __shared__ int32_t s_flag, s_count;
+    const int b = blockIdx.x;
+    const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+    if (threadIdx.x == 0) { s_flag = 0; s_count = 0; }
+    __syncthreads();
+    if (n < 0 || n > N || n > 0x10000) {
+        if (threadIdx.x == 0) {
+            atomicOr(status, n < 0 ? SPECA_STATUS_BAD_OFFSETS : SPECA_STATUS_TOO_MANY);
+            n_chains[b] = 0;
+        }
+        return;
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        sm[i] = 1;
+        sm[N + i] = -1;
+        const int pa = parent[base + i];
+        if (pa < -1 || pa >= i) atomicOr(&s_flag, 1);
+    }
+    __syncthreads();
+    if (s_flag) {
+        if (threadIdx.x == 0) { atomicOr(status, SPECA_STATUS_BAD_PARENT); n_chains[b] = 0; }
+        return;
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        for (int a = parent[base + i]; a >= 0; a = parent[base + a]) atomicAdd(&sm[a], 1);
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int pa = parent[base + i];
+        if (pa >= 0) atomicMax(&sm[N + pa], (sm[i] << 16) | (0xffff - i));       // largest subtree, then lowest index
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        int h = i;
+        for (;;) {
+            const int pa = parent[base + h];
+            if (pa < 0 || 0xffff - (sm[N + pa] & 0xffff) != h) break;            // h heads its chain
+            h = pa;
+        }
+        chain_head[base + i] = h;
+        if (h == i) atomicAdd(&s_count, 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) n_chains[b] = s_count;
+}
+
 // Confidence-guided pruning, step 1: one CTA per sequence selects its nodes and writes them, already
 // re-indexed, at the sequence's INPUT offset; out_offsets[b + 1] receives the count.  Scores are
 // accumulated in fp32 in node order, which adds every path root first, exactly as the definition does.
@@ -471,6 +526,14 @@ int launch_mask_to_parent(int32_t B, int32_t N, const uint8_t *mask, const int32
                           int32_t *status, cudaStream_t st)
 {
     mask_to_parent_kernel<<<B, 256, size_t(2 * N) * sizeof(int32_t), st>>>(N, mask, node_offsets, parent, status);
+    return int(cudaGetLastError());
+}
+
+int launch_chain_decompose(int32_t B, int32_t N, const int32_t *node_offsets, const int32_t *parent,
+                           int32_t *chain_head, int32_t *n_chains, int32_t *status, cudaStream_t st)
+{
+    chain_decompose_kernel<<<B, 256, size_t(2 * N) * sizeof(int32_t), st>>>(N, node_offsets, parent, chain_head, n_chains,
+                                                                         status);
     return int(cudaGetLastError());
 }
 

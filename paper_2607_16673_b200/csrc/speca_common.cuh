@@ -104,6 +104,8 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
 int launch_mask_to_parent(int32_t B, int32_t N, const uint8_t *mask, const int32_t *node_offsets, int32_t *parent,
                           int32_t *status, cudaStream_t st);
+int launch_chain_decompose(int32_t B, int32_t N, const int32_t *node_offsets, const int32_t *parent,
+                           int32_t *chain_head, int32_t *n_chains, int32_t *status, cudaStream_t st);
 int launch_prune(int32_t B, int32_t N, float tau, int32_t budget, const int32_t *node_offsets, const int32_t *parent,
                  const float *logp, int32_t *out_offsets, int32_t *out_parent, int32_t *out_index, int32_t *status,
                  cudaStream_t st);

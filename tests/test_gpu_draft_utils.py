@@ -131,3 +131,31 @@ def test_stochastic_accept_reports_bad_topology_and_accepts_nothing_there():
     speca.stochastic_accept(3, 3, t(offs), t(parent), one, one, zero, pidx[:, :3].contiguous(), plen, status)
     torch.cuda.synchronize()
     assert int(status.item()) & speca.STATUS_TOO_DEEP and plen.cpu().tolist()[0] == 0
+
+
+def test_chain_decompose_matches_the_definition():
+    """speca_chain_decompose against the oracle: chain heads and chain counts bit-exact."""
+    rng = np.random.default_rng(64)
+    parents, offs = batch(rng, 64, 1, 64)
+    parents[3] = synth.chain_parent(8)
+    parents[4] = synth.proposal_tree_parent(2, 14, 30, rng, 16)
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    parent = np.concatenate(parents).astype(np.int32)
+    T, B = int(offs[-1]), len(parents)
+    head = torch.full((T,), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    speca.chain_decompose(64, t(offs), t(parent), head, cnt, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    h_ref, c_ref = oracle.chain_decompose(offs, parent)
+    assert np.array_equal(head.cpu().numpy(), h_ref) and np.array_equal(cnt.cpu().numpy(), c_ref)
+    # bad topology: reported, zero chains, entries untouched; the neighbours are still decomposed
+    parents = [synth.chain_parent(3), np.array([-1, 1], np.int32), np.array([-1, 0, 0], np.int32)]
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    head = torch.full((8,), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((3,), -7, dtype=torch.int32, device="cuda")
+    speca.chain_decompose(64, t(offs), t(np.concatenate(parents).astype(np.int32)), head, cnt, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & speca.STATUS_BAD_PARENT
+    assert cnt.cpu().tolist() == [1, 0, 2] and head.cpu().tolist() == [0, 0, 0, -7, -7, 0, 0, 2]

@@ -10,6 +10,7 @@ routes that share nothing with oracle/gdn_oracle.c.
     row independence, relabelling by another topological order
   * acceptance: brute force over all root paths, hand cases; the stochastic rule: hand cases, min(1, p/q),
     the closed-form length distribution on chains, a level-free restatement
+  * heavy-light chains: the chains the paper prints for its example, partition / path / log-bound properties
   * byte counts printed by the paper (state, snapshots, factor buffer)
 """
 import itertools
@@ -619,6 +620,56 @@ def test_stochastic_accept_hand_cases_closed_form_and_level_formulation():
               if all(first.get(int(par[x])) == x for x in synth.root_path(par, t))]
         on.sort(key=lambda t: len(synth.root_path(par, t)))
         assert pi[b, :pl[b]].tolist() == on and pl[b] == len(on)
+
+
+def test_chain_decomposition_paper_example_and_properties():
+    """Section 4.3: heavy-light chains.  The chains printed for the paper's example; on random trees the
+    chains partition the nodes, each is a path of parent links, a chain hangs off a node of another chain (or
+    the committed state), and a root path changes chain at most floor(log2 n) times (the property that
+    makes the policy "heavy-light")."""
+    parent, chains = {}, []
+    for line in open(os.path.join(GOLDEN, "hld_example.txt")):
+        tok = line.split()
+        if not tok or tok[0].startswith("#"):
+            continue
+        if tok[0] == "parent":
+            parent = {int(a.split(":")[0]): int(a.split(":")[1]) for a in tok[1:]}
+        elif tok[0] == "chain":
+            chains.append([int(x) for x in tok[1:]])
+    n = len(parent)
+    par = np.array([parent[i + 1] - 1 for i in range(n)], np.int32)          # 1-based, 0 = committed state -> local, -1
+    head, cnt = oracle.chain_decompose(np.array([0, n], np.int32), par)
+    got = {}
+    for t in range(n):
+        got.setdefault(int(head[t]) + 1, []).append(t + 1)
+    assert sorted(got.values()) == sorted(chains) and cnt.tolist() == [len(chains)]
+    # hand case with a tie and a forest: 0 -> {1, 2} (equal subtrees: the lower index is heavy), second root 3
+    head, cnt = oracle.chain_decompose(np.array([0, 5], np.int32), np.array([-1, 0, 0, -1, 3], np.int32))
+    assert head.tolist() == [0, 0, 2, 3, 3] and cnt.tolist() == [3]
+    rng = np.random.default_rng(91)
+    parents = [synth.random_tree_parent(int(rng.integers(1, 65)), 8, 4, rng) for _ in range(40)]
+    parents += [synth.chain_parent(8), np.zeros(0, np.int32), synth.proposal_tree_parent(2, 14, 30, rng, 16)]
+    offs = np.concatenate([[0], np.cumsum([len(pp) for pp in parents])]).astype(np.int32)
+    head, cnt = oracle.chain_decompose(offs, np.concatenate(parents).astype(np.int32))
+    for b, par in enumerate(parents):
+        n = len(par)
+        h = head[offs[b]:offs[b + 1]]
+        members = {}
+        for t in range(n):
+            members.setdefault(int(h[t]), []).append(t)
+        assert cnt[b] == len(members) and all(k == v[0] for k, v in members.items())
+        size = [len([t for t in range(n) if i in synth.root_path(par, t)]) for i in range(n)]      # brute force
+        for k, v in members.items():
+            for a_, b_ in zip(v, v[1:]):
+                assert par[b_] == a_                                                      # a path of parent links
+                sib = [t for t in range(n) if par[t] == a_]
+                assert size[b_] == max(size[t] for t in sib)                               # along the heaviest child
+                assert b_ == min(t for t in sib if size[t] == size[b_])                    # lowest index on ties
+            assert par[k] < 0 or h[par[k]] != k                                           # the head hangs off another chain
+        for t in range(n):
+            path = synth.root_path(par, t)
+            changes = sum(1 for a_, b_ in zip(path, path[1:]) if h[a_] != h[b_])
+            assert changes <= int(np.floor(np.log2(n)))
 
 
 def test_rule_without_erase_is_gated_linear_attention():
