@@ -92,7 +92,7 @@ def test_stochastic_accept_matches_the_walk():
         parent = np.concatenate(parents).astype(np.int32)
         T = int(offs[-1])
         p_draft = rng.uniform(0.02, 1.0, T).astype(np.float32)
-        # ratios p/q spread around 1 so that paths of every length occur; some exact ties u * q == p
+        # ratios p/q on both sides of one, so that paths of every length occur; some exact ties u * q == p
         p_target = (p_draft * rng.choice([0.25, 0.5, 1.0, 2.0], T)).astype(np.float32)
         uniform = rng.random(T, dtype=np.float32)
         ties = rng.random(T) < 0.05
