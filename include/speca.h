@@ -85,10 +85,16 @@ extern "C" {
 /* verification routes (dims.route) */
 #define SPECA_ROUTE_AUTO        0   /* library picks                                              */
 #define SPECA_ROUTE_SERIAL      1   /* state-resident walk, one rank-1 update per node (Section 4.1) */
-#define SPECA_ROUTE_FACTORIZED  2   /* tree-masked WY form on tensor cores (Section 4.2)           */
-/* The tensor-core route takes d_v in {128, 256} and: max_depth <= 8 with max_nodes <= 64 (d_k = 128) or <= 32
- * (d_k = 256); 8 < max_depth <= 16 with max_nodes <= 32 (d_k = 128 or 256).  AUTO uses it whenever it applies
- * and the serial route otherwise; asking for it explicitly outside these shapes is SPECA_ERR_UNSUPPORTED. */
+#define SPECA_ROUTE_FACTORIZED  2   /* tree-masked factorised form on tensor cores (Section 4.2), fp32-grade */
+#define SPECA_ROUTE_TF32        3   /* the same factorisation with the state read once as TF32 (single pass)  */
+/* SPECA_ROUTE_FACTORIZED takes d_v in {128, 256}, max_depth <= 16 and max_nodes <= 64 (d_k = 128) or <= 32
+ * (d_k = 256).  Both tensor-core operands are split into a TF32 head and its exact remainder, so outputs
+ * carry fp32 accuracy whatever the magnitude of the state.  AUTO uses it whenever it applies and the serial
+ * route otherwise; asking for it explicitly outside these shapes is SPECA_ERR_UNSUPPORTED.
+ * SPECA_ROUTE_TF32 is never picked by AUTO: it reads the fp32 state through a single TF32 pass (10 mantissa
+ * bits, truncated), which leaves errors of about 2^-11 of the output's scale, growing with the state; it takes
+ * max_depth <= 8 with max_nodes <= 64 (d_k = 128) or <= 32 (d_k = 256), or max_depth <= 16 with max_nodes <=
+ * 32, and is the only route on which speca_commit_verify_tree runs as ONE pass over the state. */
 
 /* recurrences (dims.rule; Section 5.1, remark on other layer types).  A DeltaNet layer (k, v, beta, no
  * decay) is the gated delta rule with alpha = 1 and needs no value of its own. */

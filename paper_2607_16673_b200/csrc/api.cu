@@ -15,7 +15,7 @@ int check_dims(const speca_dims *d)
     if (d->d_v < 32 || d->d_v > 1024 || d->d_v % 32 != 0) return SPECA_ERR_UNSUPPORTED;
     if (d->max_depth < 1 || d->max_depth > 16) return SPECA_ERR_RANGE;
     if (d->max_nodes < 1 || d->max_nodes > 1024) return SPECA_ERR_RANGE;
-    if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_FACTORIZED) return SPECA_ERR_UNSUPPORTED;
+    if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_TF32) return SPECA_ERR_UNSUPPORTED;
     if (d->rule != SPECA_RULE_GATED_DELTA && d->rule != SPECA_RULE_GATED_NO_ERASE) return SPECA_ERR_UNSUPPORTED;
     const long long units = 1LL * d->n_layers * d->batch * d->heads;
     if (units * (d->d_v / 2) > 0x7fffffffLL) return SPECA_ERR_RANGE;       // grid size bound
@@ -65,15 +65,20 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
     p.status = status_word;
     p.ws = carve_workspace(workspace, dims->batch, total_nodes);
     p.n_slots = tree_slots_needed(dims->max_nodes);
-    const bool can_factorize = factorized_supported(dims);
-    if (dims->route == SPECA_ROUTE_FACTORIZED && !can_factorize) return SPECA_ERR_UNSUPPORTED;
-    const bool factorize = can_factorize && dims->route != SPECA_ROUTE_SERIAL;
-    if (!chain || factorize) {
+    // AUTO: the fp32-grade tensor-core route where the shape fits, else the serial walk.  The single-pass
+    // TF32 kernel runs only when asked for by name.
+    const bool tf32 = dims->route == SPECA_ROUTE_TF32;
+    if (tf32 && !factorized_supported(dims)) return SPECA_ERR_UNSUPPORTED;
+    const bool can_eff = effective_supported(dims);
+    if (dims->route == SPECA_ROUTE_FACTORIZED && !can_eff) return SPECA_ERR_UNSUPPORTED;
+    const bool eff = can_eff && (dims->route == SPECA_ROUTE_AUTO || dims->route == SPECA_ROUTE_FACTORIZED);
+    if (!chain || eff || tf32) {
         // with parent == NULL (chain entry point) the plan kernel assumes parent[i] = i - 1
         rc = cuda_rc(launch_plan(p, st));
         if (rc != SPECA_OK) return rc;
     }
-    if (factorize) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, st));
+    if (eff) return cuda_rc(launch_verify_effective(p, dims->d_k, st));
+    if (tf32) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, st));
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 
@@ -302,10 +307,10 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k
     if (total_nodes > 0 && workspace_bytes < speca::workspace_bytes(dims->batch, total_nodes))
         return SPECA_ERR_WORKSPACE;
 
-    // One pass over the state when the tensor-core route applies and the previous verification
-    // left its u; otherwise the two kernels run back to back on the stream (same results).
+    // One pass over the state on the single-pass TF32 route, when the previous verification left its
+    // u; otherwise the commit and verify kernels run back to back on the stream (same results, fp32-grade).
     const bool one_pass = have_commit && total_nodes > 0 && u_prev_or_null != nullptr && factorized_fused_supported(dims) &&
-                          dims->route != SPECA_ROUTE_SERIAL;
+                          dims->route == SPECA_ROUTE_TF32;
     if (!one_pass) {
         if (have_commit) {
             rc = speca_commit(dims, S, k_prev, v_prev, alpha_prev, beta_prev, node_offsets_prev, total_nodes_prev,

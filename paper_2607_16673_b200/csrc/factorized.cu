@@ -46,10 +46,13 @@
 #include <type_traits>
 
 #include "speca_common.cuh"
+#include "tc_ptx.cuh"
 
 namespace speca {
 
 namespace {
+
+using namespace tc;
 
 constexpr int kDK = 128;                       // key width handled by this route
 constexpr int kTileRows = 128;                 // value rows per tile (= TMEM lanes = MMA M)
@@ -129,76 +132,6 @@ enum Bar {
 };
 static_assert(kBarCount <= 40, "barrier region too small");
 
-// ----------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// non-blocking probe of a barrier phase
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_timer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded, warp-uniform wait.  Returns false if the CTA is aborting (this wait or another
-// one gave up); the caller must then leave its loop.  All 32 lanes must call it together.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;       // 2 s
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    uint64_t t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        const bool ok = mbar_try_wait(bar, parity);
-        if (__any_sync(0xffffffffu, ok)) return true;
-#ifdef SPECA_SPIN_SLEEP
-        __nanosleep(SPECA_SPIN_SLEEP);
-#endif
-        if ((it & 255u) == 255u) {
-            if (__any_sync(0xffffffffu, *abort_flag != 0)) return false;
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            if (__any_sync(0xffffffffu, now - t0 > kWaitLimitNs)) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-}
 
 // Optional self-profiling build (-DSPECA_PROF): cycles spent in each kind of wait per role.
 #ifdef SPECA_PROF
@@ -228,116 +161,6 @@ __device__ __forceinline__ bool prof_wait(long long &acc, uint32_t bar, uint32_t
 #define PROF_STORE()
 #endif
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-        : "memory");
-}
-// bring a box of a tensor into L2 ahead of the loads that will use it (no destination, no barrier)
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int x, int y, int z)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
-                 : "memory");
-}
-// untiled bulk copy global -> shared (both addresses and the size multiples of 16 bytes)
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_3d_nocommit(const CUtensorMap *map, int x, int y, int z, uint32_t src)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src)
-                 : "memory");
-}
-// all but the newest N store groups have finished READING shared memory
-template <int N> __device__ __forceinline__ void tma_store_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-// every store group has completed
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async()
-{
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&r)[8])
-{
-    uint32_t x[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]), "=r"(x[7])
-                 : "r"(taddr)
-                 : "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) r[i] = __uint_as_float(x[i]);
-}
-__device__ __forceinline__ void tmem_ld4(uint32_t taddr, float (&r)[4])
-{
-    uint32_t x[4];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
-                 : "r"(taddr)
-                 : "memory");
-#pragma unroll
-    for (int i = 0; i < 4; ++i) r[i] = __uint_as_float(x[i]);
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major operand descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
-{
-    uint64_t d = 0;
-    d |= uint64_t((smem_addr >> 4) & 0x3fffu);          // start address
-    d |= uint64_t(1) << 16;                              // leading byte offset (unused for swizzled K-major)
-    d |= uint64_t(1024 >> 4) << 32;                      // stride byte offset between 8-row groups
-    d |= uint64_t(1) << 46;                              // descriptor version (Blackwell)
-    d |= uint64_t(2) << 61;                              // SWIZZLE_128B
-    return d;
-}
-// warp-level D = A B + D, m16n8k8, TF32 operands (bit patterns), fp32 accumulate
-__device__ __forceinline__ void mma_tf32_sync(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-                 "{%0, %1, %2, %3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// kind::tf32, fp32 accumulate, both operands K-major, M = 128
-__device__ __forceinline__ uint32_t make_idesc(int n)
-{
-    return (1u << 4) | (2u << 7) | (2u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(kTileRows >> 4) << 24);
-}
 
 // Tensor maps of the bf16 key / query records, view [L*T][H][d_k], one per box height
 // (16, 32, 48, 64 nodes): a unit's rows are fetched with the smallest box that covers them.
@@ -361,21 +184,6 @@ __device__ __forceinline__ int anc_byte16(const int4 &meta, int meta2, int j)
     return int((w >> (8 * (j & 3))) & 0xffu);
 }
 
-// kind::f16 with bf16 operands, fp32 accumulate, both operands K-major, M = 128 (Gram block)
-__device__ __forceinline__ uint32_t make_idesc_bf16(int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(kTileRows >> 4) << 24);
-}
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
 
 // Units are taken in groups of HG consecutive heads of one (layer, sequence): group
 // G = blockIdx.x, += gridDim.x.  Inside a group the topology-dependent data (node count,
@@ -429,12 +237,6 @@ __device__ __forceinline__ bool next_unit(const UnitWalk &w, Unit &x)
     return load_group(w, x.grp + w.grid, x);
 }
 
-// try once inline; fall into the bounded polling loop only if the barrier is not ready yet
-__device__ __forceinline__ bool wait_fast(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-    return mbar_wait(bar, parity, abort_flag);
-}
 
 // One node of the forward substitution for TP value rows (one per tile of the unit),
 // branch-free.  The u of the nodes on the current depth-first path live in ustk[.][depth-1];
@@ -1400,22 +1202,6 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            sym = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(sym);
-    }();
-    return fn;
-}
 
 }  // namespace
 

@@ -101,6 +101,9 @@ int launch_commit(const Params &p, int d_k, cudaStream_t st);
 bool factorized_supported(const speca_dims *d);
 bool factorized_fused_supported(const speca_dims *d);
 int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st);
+bool effective_supported(const speca_dims *d);
+int launch_verify_effective(const Params &p, int d_k, cudaStream_t st);
+void effective_set_withhold(int on);
 int launch_pending_check(const Params &p, int max_len, cudaStream_t st);
 int launch_mask_to_parent(int32_t B, int32_t N, const uint8_t *mask, const int32_t *node_offsets, int32_t *parent,
                           int32_t *status, cudaStream_t st);
