@@ -53,7 +53,6 @@ constexpr int kAccCols = 128;                   // accumulator columns per tile:
 constexpr int kPairCols = 2 * kAccCols;
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 18 * 32;
-constexpr int kPrepThreads = 256;
 constexpr int kSolveThreads = 128;
 constexpr int kSplitThreads = 128;
 constexpr int kRecBytes = 112;                  // per operand row: count, 17 weights, 17 staging offsets
@@ -71,7 +70,9 @@ template <int TP, int DK> struct Lay {
     static constexpr int MPIECE = MAXN * 128;                   // one bf16 piece of M: R rows x 64 columns
     static constexpr int VBLK = MAXN * 128;                     // 64 values of all nodes
     static constexpr int VBYTES = TP * 2 * VBLK;
-    static constexpr int kFixed = 2 * BBUF + 2 * STAGE + 3 * MPIECE + VBYTES + 64 * kRecBytes + 2 * 64 * 4 + 512 + 64 +
+    static constexpr int kTemp = MAXN * kRows * 4;              // whole Gram block of a unit, parked in the value-row buffer
+    static constexpr int VREG = VBYTES > kTemp ? VBYTES : kTemp;
+    static constexpr int kFixed = 2 * BBUF + 2 * STAGE + 3 * MPIECE + VREG + 64 * kRecBytes + 2 * 64 * 4 + 512 + 64 +
                                   5 * kWalkSeqs;
     static constexpr int kRoom = (227 * 1024 - kFixed - 1024) / kSliceBytes;
     static constexpr int NS = kRoom > 6 ? 6 : kRoom;            // ring depth
@@ -80,7 +81,8 @@ template <int TP, int DK> struct Lay {
     static constexpr int OffStage = OffB + 2 * BBUF;
     static constexpr int OffM = OffStage + 2 * STAGE;
     static constexpr int OffV = OffM + 3 * MPIECE;
-    static constexpr int OffRec = OffV + VBYTES;                // Gram scratch, then X rows, then records
+    static constexpr int OffTemp = OffV;
+    static constexpr int OffRec = OffV + VREG;
     static constexpr int OffAlpha = OffRec + 64 * kRecBytes;
     static constexpr int OffBars = OffAlpha + 2 * 64 * 4;
     static constexpr int OffMisc = OffBars + 512;
@@ -88,7 +90,6 @@ template <int TP, int DK> struct Lay {
     static constexpr int Bytes = OffWalk + 5 * kWalkSeqs;
     static_assert(NS >= 4, "ring too shallow");
     static_assert(Bytes <= 227 * 1024, "shared memory budget");
-    static_assert(64 * kRecBytes >= 8 * kRows * 4 && 64 * kRecBytes >= MAXN * kMaxD * 4, "scratch aliases");
 };
 
 enum Bar {
@@ -107,8 +108,10 @@ enum Bar {
     kVFree,                    // MMA -> prep (which issues the copy)
     kAccFull,                  // [2] MMA -> epilogue
     kPairFree = kAccFull + 2,  // [2] epilogue -> MMA
-    kPrepSync = kPairFree + 2, // prep-internal
-    kSolveSync,
+    kRecReady = kPairFree + 2, // solver -> vector warps: records of a unit written
+    kRecFree,                  // vector warps -> solver
+    kSolveSync,                // role-internal
+    kVecSync,
     kDrain,
     kBarCount
 };
@@ -168,8 +171,44 @@ __device__ __forceinline__ int anc_at(const int4 &meta, int meta2, int j)
     return int((w >> (8 * (j & 3))) & 0xffu);
 }
 
+// one arrival for the whole warp: every lane's earlier writes are ordered before it
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+
+// Optional self-profiling build (-DSPECA_PROF): cycles CTA 0 spends in each kind of wait, per warp,
+// written to the control words of the workspace ([8 + 9 warp .. ): 8 slots and the warp's lifetime).
+#ifdef SPECA_PROF
+#define PROF_DECL long long prof_w[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long prof_t0 = clock64();
+#define WAIT(slot, b, ph) prof_wait(prof_w[slot], b, ph, abort_flag)
+#define PROF_T0() const long long prof_seg0 = clock64();
+#define PROF_ADD(slot) prof_w[slot] += clock64() - prof_seg0;
+#define PROF_STORE()                                                                              \
+    if (blockIdx.x == 0 && lane == 0) {                                                           \
+        long long *dst = reinterpret_cast<long long *>(p.ws.ctrl) + 8 + warp * 9;                \
+        for (int i_ = 0; i_ < 8; ++i_) dst[i_] = prof_w[i_];                                      \
+        dst[8] = clock64() - prof_t0;                                                             \
+    }
+__device__ __forceinline__ bool prof_wait(long long &acc, uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    const long long t = clock64();
+    const bool r = wait_fast(bar, parity, abort_flag);
+    acc += clock64() - t;
+    return r;
+}
+#else
+#define PROF_DECL
+#define PROF_T0()
+#define PROF_ADD(slot)
+#define WAIT(slot, b, ph) wait_fast(b, ph, abort_flag)
+#define PROF_STORE()
+#endif
 
 // TP = value tiles per unit (d_v / 128), DK = key width.
 template <int TP, int DK>
@@ -197,23 +236,25 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
             mbar_init(bar(kFull + s), 1);
             mbar_init(bar(kEmpty + s), 1);
             mbar_init(bar(kP1Done + s), 1);
-            mbar_init(bar(kLo + s), kSplitThreads);
+            mbar_init(bar(kLo + s), kSplitThreads / 32);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kKQFull + i), 1);
-            mbar_init(bar(kBReady + i), kPrepThreads);
+            mbar_init(bar(kBReady + i), 4);
             mbar_init(bar(kBFree + i), 1);
             mbar_init(bar(kAccFull + i), 1);
-            mbar_init(bar(kPairFree + i), 128);
+            mbar_init(bar(kPairFree + i), 4);
         }
         mbar_init(bar(kGramFull), 1);
-        mbar_init(bar(kGramDone), kSolveThreads);
-        mbar_init(bar(kMReady), kSolveThreads);
+        mbar_init(bar(kGramDone), kSolveThreads / 32);
+        mbar_init(bar(kMReady), kSolveThreads / 32);
         mbar_init(bar(kMFree), 1);
         mbar_init(bar(kVFull), 1);
         mbar_init(bar(kVFree), 1);
-        mbar_init(bar(kPrepSync), kPrepThreads);
-        mbar_init(bar(kSolveSync), kSolveThreads);
+        mbar_init(bar(kRecReady), 4);
+        mbar_init(bar(kRecFree), 4);
+        mbar_init(bar(kSolveSync), 4);
+        mbar_init(bar(kVecSync), 4);
         mbar_init(bar(kDrain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -241,11 +282,12 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
         uint32_t it = 0;
         VUnit x;
         bool ok = true;
+        PROF_DECL
         for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
             for (int c = 0; c < NC && ok; ++c) {
                 for (int t = 0; t < TP; ++t, ++it) {
                     const int s = it % NS;
-                    if (!(ok = wait_fast(bar(kEmpty + s), ((it / NS) & 1) ^ 1, abort_flag))) break;
+                    if (!(ok = WAIT(0, bar(kEmpty + s), ((it / NS) & 1) ^ 1))) break;
                     if (lane == 0 && !(ep.withhold_first_load && blockIdx.x == 0 && it == 0)) {
                         mbar_arrive_expect_tx(bar(kFull + s), kSliceBytes);
                         tma_load_3d(sbase + LY::OffRing + s * kSliceBytes, &s0_map, c * 32, t * kRows, x.u, bar(kFull + s));
@@ -254,6 +296,7 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                 }
             }
         }
+        PROF_STORE()
         // let copies still in flight land before the CTA's shared memory goes away
         if (*abort_flag) {
             const uint64_t t0 = global_timer_ns();
@@ -261,39 +304,28 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        uint32_t it = 0, useq = 0, cc = 0;
-        VUnit x, nx;
-        bool ok = true;
-        // second pass of the slice issued last: waits for its remainder, then releases what the slice held
-        bool pend = false;
-        uint32_t pend_slot = 0, pend_b = 0, pend_acc = 0, pend_id = 0, pend_ph = 0;
-        int pend_s = 0, pend_bfree = -1, pend_accfull = -1;
-        auto flush_pend = [&]() -> bool {
-            if (!wait_fast(bar(kLo + pend_s), pend_ph, abort_flag)) return false;
-            tc_fence_after();
-            if (lane == 0) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    mma_tf32(pend_acc, make_desc(pend_slot + k * 32), make_desc(pend_b + k * 32), pend_id, 1);
-                mma_commit(bar(kEmpty + pend_s));
-                if (pend_bfree >= 0) mma_commit(bar(kBFree + pend_bfree));
-                if (pend_accfull >= 0) mma_commit(bar(kAccFull + pend_accfull));
+        // Two cursors walk the same sequence of slices: the first pass is issued as soon as a slice and its
+        // operand have landed, the second pass as soon as the slice has been rewritten as its remainder.
+        // Neither blocks the other: the warp polls and serves whichever is ready.
+        struct Cur { VUnit x; uint32_t useq, it, cc; int c, t; bool have; };
+        auto advance = [&](Cur &q) {
+            ++q.it;
+            if (++q.t == TP) {
+                q.t = 0; ++q.cc;
+                if (++q.c == NC) { q.c = 0; ++q.useq; q.have = next_unit(walk, q.x); }
             }
-            __syncwarp();
-            pend = false;
-            return true;
         };
+        bool ok = true;
+        PROF_DECL
         // Gram block of a unit: [K;Q] (128 rows) x K^T (npad columns) from the staged bf16 rows, parked in the
-        // unit's own accumulator columns until its state MMAs overwrite them.  1 issued, 0 not yet, -1 abort.
-        auto issue_gram = [&](uint32_t seq, int npad, bool blocking) -> int {
+        // unit's own accumulator columns until its state MMAs overwrite them.
+        auto gram_ready = [&](uint32_t seq) -> bool {
             const int pr = seq & 1;
-            const uint32_t bk = bar(kKQFull + pr), pk = (seq >> 1) & 1;
-            const uint32_t bp = bar(kPairFree + pr), pp = ((seq >> 1) & 1) ^ 1;
-            if (blocking) {
-                if (!wait_fast(bk, pk, abort_flag) || !wait_fast(bp, pp, abort_flag)) return -1;
-            } else if (!__all_sync(0xffffffffu, mbar_test_wait(bk, pk) && mbar_test_wait(bp, pp))) {
-                return 0;
-            }
+            return __all_sync(0xffffffffu, mbar_test_wait(bar(kKQFull + pr), (seq >> 1) & 1) &&
+                                               mbar_test_wait(bar(kPairFree + pr), ((seq >> 1) & 1) ^ 1));
+        };
+        auto issue_gram = [&](uint32_t seq, int npad) {
+            const int pr = seq & 1;
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t idg = make_idesc_bf16(npad);
@@ -308,101 +340,294 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                 mma_commit(bar(kGramFull));
             }
             __syncwarp();
-            return 1;
         };
-        bool have = first_unit(walk, x);
-        if (have) ok = issue_gram(0, x.npad, true) > 0;
-        while (have && ok) {
-            const int pr = useq & 1;
-            const uint32_t acc = tmem_base + pr * kPairCols;
-            const int R = x.npad;
-            nx = x;
-            const bool have_next = next_unit(walk, nx);
-            bool gram_issued = !have_next;
-            if (!(ok = wait_fast(bar(kGramDone), useq & 1, abort_flag))) break;
-            tc_fence_after();
-            const uint32_t id1 = make_idesc(2 * R), id2 = make_idesc(R);
-            for (int c = 0; c < NC && ok; ++c, ++cc) {
-                const int bb = cc & 1;
-                if (!(ok = wait_fast(bar(kBReady + bb), (cc >> 1) & 1, abort_flag))) break;
-                const uint32_t ba = sbase + LY::OffB + bb * LY::BBUF;
-                for (int t = 0; t < TP && ok; ++t, ++it) {
-                    const int s = it % NS;
-                    if (!(ok = wait_fast(bar(kFull + s), (it / NS) & 1, abort_flag))) break;
+        Cur c1, c2;
+        c1.useq = c1.it = c1.cc = 0; c1.c = c1.t = 0;
+        c1.have = first_unit(walk, c1.x);
+        c2 = c1;
+        VUnit nx = c1.x;
+        bool have_next = c1.have && next_unit(walk, nx);
+        uint32_t gram_seq = 0;                                   // Gram blocks issued so far
+        uint64_t t0 = 0;
+        uint32_t spin = 0;
+        while (ok && (c1.have || c2.it < c1.it)) {
+            bool prog = false;
+            // the Gram block of the unit the first cursor is in, or of the one after it
+            if (c1.have && gram_seq == c1.useq && gram_ready(gram_seq)) {
+                issue_gram(gram_seq, c1.x.npad);
+                ++gram_seq;
+                prog = true;
+            } else if (c1.have && have_next && gram_seq == c1.useq + 1 && (c1.c > 0 || c1.t > 0) && gram_ready(gram_seq)) {
+                issue_gram(gram_seq, nx.npad);
+                ++gram_seq;
+                prog = true;
+            }
+            // second pass
+            if (c2.it < c1.it) {
+                const int s = c2.it % NS;
+                if (__all_sync(0xffffffffu, mbar_test_wait(bar(kLo + s), (c2.it / NS) & 1))) {
                     tc_fence_after();
-                    const uint32_t sa = sbase + LY::OffRing + s * kSliceBytes;
                     if (lane == 0) {
+                        const uint32_t sa = sbase + LY::OffRing + s * kSliceBytes;
+                        const uint32_t ba = sbase + LY::OffB + (c2.cc & 1) * LY::BBUF;
+                        const uint32_t acc = tmem_base + (c2.useq & 1) * kPairCols + c2.t * kAccCols;
+                        const uint32_t id2 = make_idesc(c2.x.npad);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            mma_tf32(acc + t * kAccCols, make_desc(sa + k * 32), make_desc(ba + k * 32), id1, (c | k) != 0);
-                        mma_commit(bar(kP1Done + s));
+                        for (int k = 0; k < 4; ++k) mma_tf32(acc, make_desc(sa + k * 32), make_desc(ba + k * 32), id2, 1);
+                        mma_commit(bar(kEmpty + s));
+                        if (c2.t == TP - 1) mma_commit(bar(kBFree + (c2.cc & 1)));
+                        if (c2.t == TP - 1 && c2.c == NC - 1) mma_commit(bar(kAccFull + (c2.useq & 1)));
                     }
                     __syncwarp();
-                    if (c == 0) {
-                        // value term of this tile: V^T (128 values x R nodes, as landed) x M^T, three bf16 pieces
-                        if (t == 0) {
-                            if (!(ok = wait_fast(bar(kMReady), useq & 1, abort_flag))) break;
-                            if (!(ok = wait_fast(bar(kVFull), useq & 1, abort_flag))) break;
-                            tc_fence_after();
-                        }
-                        if (lane == 0) {
+                    advance(c2);
+                    prog = true;
+                }
+            }
+            // first pass
+            if (c1.have && gram_seq > c1.useq) {
+                const int s = c1.it % NS;
+                bool ready = mbar_test_wait(bar(kBReady + (c1.cc & 1)), (c1.cc >> 1) & 1) &&
+                             mbar_test_wait(bar(kFull + s), (c1.it / NS) & 1);
+                if (c1.c == 0 && c1.t == 0) ready = ready && mbar_test_wait(bar(kGramDone), c1.useq & 1);
+                if (c1.c == 1 && c1.t == 0)
+                    ready = ready && mbar_test_wait(bar(kMReady), c1.useq & 1) && mbar_test_wait(bar(kVFull), c1.useq & 1);
+                // the last slice of a unit waits for the next unit's Gram block to be on its way, so that the
+                // preparation of that unit is never queued behind a whole unit of state MMAs
+                if (c1.c == NC - 1 && c1.t == TP - 1 && have_next && gram_seq < c1.useq + 2) ready = false;
+                if (__all_sync(0xffffffffu, ready)) {
+                    tc_fence_after();
+                    const int R = c1.x.npad;
+                    const uint32_t acc = tmem_base + (c1.useq & 1) * kPairCols + c1.t * kAccCols;
+                    if (lane == 0) {
+                        const uint32_t sa = sbase + LY::OffRing + s * kSliceBytes;
+                        const uint32_t ba = sbase + LY::OffB + (c1.cc & 1) * LY::BBUF;
+                        const uint32_t id1 = make_idesc(2 * R);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_tf32(acc, make_desc(sa + k * 32), make_desc(ba + k * 32), id1, (c1.c | k) != 0);
+                        mma_commit(bar(kP1Done + s));
+                        if (c1.c == 1) {
+                            // value term of this tile: V^T (128 values x R nodes, as landed) x M^T, three bf16 pieces
                             const uint32_t idv = make_idesc_bf16_amn(R);
-                            const uint32_t vb = sbase + LY::OffV + t * 2 * LY::VBLK, mb = sbase + LY::OffM;
+                            const uint32_t vb = sbase + LY::OffV + c1.t * 2 * LY::VBLK, mb = sbase + LY::OffM;
                             for (int piece = 0; piece < 3; ++piece)
                                 for (int ks = 0; ks < R / 16; ++ks)
-                                    mma_bf16(acc + t * kAccCols, make_desc_mn(vb + ks * 2048, LY::VBLK),
+                                    mma_bf16(acc, make_desc_mn(vb + ks * 2048, LY::VBLK),
                                              make_desc(mb + piece * LY::MPIECE + ks * 32), idv, 1);
-                            if (t == TP - 1) { mma_commit(bar(kVFree)); mma_commit(bar(kMFree)); }
+                            if (c1.t == TP - 1) { mma_commit(bar(kVFree)); mma_commit(bar(kMFree)); }
                         }
-                        __syncwarp();
                     }
-                    if (pend && !(ok = flush_pend())) break;
-                    pend = true;
-                    pend_slot = sa; pend_b = ba; pend_acc = acc + t * kAccCols; pend_id = id2;
-                    pend_s = s; pend_ph = (it / NS) & 1;
-                    pend_bfree = (t == TP - 1) ? bb : -1;
-                    pend_accfull = (c == NC - 1 && t == TP - 1) ? pr : -1;
+                    __syncwarp();
+                    const uint32_t was = c1.useq;
+                    advance(c1);
+                    if (c1.useq != was) {
+                        nx = c1.x;
+                        have_next = c1.have && next_unit(walk, nx);
+                    }
+                    prog = true;
                 }
-                if (ok && !gram_issued && c >= 1) {
-                    const int r = issue_gram(useq + 1, nx.npad, c == NC - 1);
-                    if (r < 0) ok = false;
-                    else gram_issued = r > 0;
+            }
+            if (prog) {
+                spin = 0; t0 = 0;
+            } else {
+                __nanosleep(20);
+                if ((++spin & 255u) == 0u) {
+                    if (__any_sync(0xffffffffu, *abort_flag != 0)) ok = false;
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    if (__any_sync(0xffffffffu, now - t0 > kWaitLimitNs)) { *abort_flag = 1; ok = false; }
                 }
+            }
+        }
+        PROF_STORE()
+        // everything this warp issued must have completed before TMEM is released
+        if (lane == 0) mma_commit(bar(kDrain));
+        __syncwarp();
+        mbar_wait(bar(kDrain), 0, abort_flag);
+    } else if (warp < 6) {
+        // ------------------------------------------------------------- solver: Gram block -> records and M
+        const int stid = threadIdx.x - 64;                       // 0..127
+        const int grow = 32 * (warp & 3) + lane;                 // Gram row (= TMEM lane) of this thread
+        const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
+        float *G = reinterpret_cast<float *>(smem + LY::OffTemp);   // whole Gram block, [column][128 rows]
+        uint8_t *rec = smem + LY::OffRec;
+        float *alpha_s = reinterpret_cast<float *>(smem + LY::OffAlpha);
+        float *beta_s = alpha_s + 64;
+        uint32_t ssync = 0, useq = 0;
+        PROF_DECL
+        auto solve_sync = [&]() -> bool {
+            warp_arrive(bar(kSolveSync), lane);
+            const bool r = WAIT(0, bar(kSolveSync), ssync & 1);
+            ++ssync;
+            return r;
+        };
+        // per-thread topology and gates of a unit, fetched one unit ahead
+        int4 meta_n = make_int4(0, 0, 0, 0);
+        int meta2_n = 0;
+        float alpha_n = 0.f, beta_n = 0.f;
+        auto fetch_topo = [&](const VUnit &y) {
+            const int node = grow < y.npad ? grow : grow - y.npad;
+            const bool act = grow < 2 * y.npad && node < y.n;
+            meta_n = act ? __ldg(reinterpret_cast<const int4 *>(p.ws.anc) + y.base + node) : make_int4(0, 0, 0, 0);
+            meta2_n = act ? __ldg(p.ws.anc2 + 4 * (y.base + node)) : 0;
+            if (stid < y.n) {
+                const int r = (y.l * p.T + y.base + stid) * p.H + y.h;
+                alpha_n = __ldg(p.alpha + r);
+                beta_n = __ldg(p.beta + r);
+            }
+        };
+        VUnit x, nx;
+        bool ok = true;
+        bool have = first_unit(walk, x);
+        if (have) fetch_topo(x);
+        while (have && ok) {
+            const int R = x.npad;
+            const int4 meta = meta_n;
+            const int meta2 = meta2_n;
+            const float my_alpha = alpha_n, my_beta = beta_n;
+            nx = x;
+            const bool have_next = next_unit(walk, nx);
+            if (have_next) fetch_topo(nx);
+            // ancestors by level, one byte each
+            const unsigned long long anc_lo = (unsigned long long)(uint32_t(meta.y)) | ((unsigned long long)(uint32_t(meta.z)) << 32);
+            const unsigned long long anc_hi = (unsigned long long)(uint32_t(meta.w)) | ((unsigned long long)(uint32_t(meta2)) << 32);
+            const bool is_k = grow < R;
+            const int node = is_k ? grow : grow - R;
+            const bool in_rows = grow < 2 * R;
+            const bool active = in_rows && node < x.n;
+            const int d = active ? (meta.x & 0xff) : 0;
+            auto anc = [&](int j) -> int {
+                const int a = int(((j < 8 ? anc_lo : anc_hi) >> (8 * (j & 7))) & 0xffull);
+                return j < d - 1 ? a : node;
+            };
+            // The scratch below sits in the value-row buffer: the previous unit's value term must have read it.
+            if (!(ok = WAIT(2, bar(kVFree), (useq & 1) ^ 1))) break;
+            if (!(ok = WAIT(4, bar(kGramFull), useq & 1))) break;
+            tc_fence_after();
+            PROF_T0()
+            {
+                // whole Gram row of this thread -> G[column][row]
+                const uint32_t gaddr = tmem_base + (useq & 1) * kPairCols + lane_addr;
+#pragma unroll 1
+                for (int c0 = 0; c0 < R; c0 += 16) {
+                    float t8[8], u8[8];
+                    tmem_ld8(gaddr + c0, t8);
+                    tmem_ld8(gaddr + c0 + 8, u8);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) G[(c0 + i) * kRows + grow] = t8[i];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) G[(c0 + 8 + i) * kRows + grow] = u8[i];
+                }
+                tc_fence_before();
+                warp_arrive(bar(kGramDone), lane);               // the state MMAs may now overwrite these columns
+            }
+            if (stid < x.n) { alpha_s[stid] = my_alpha; beta_s[stid] = my_beta; }
+            PROF_ADD(1)
+            if (!(ok = solve_sync())) break;                     // Gram block and gates visible
+
+            // Row of X = (I + Ahat)^-1 (key rows, right-hand side e_t) or of C = Phat X (query rows, right-hand
+            // side the row's own q.k entries) by back substitution along the path:
+            //     c_j = rhs_j - sum_{m > j} c_m beta_{a_m} (k_{a_m} . k_{a_j}).
+            float cf[kMaxD];
+            {
+                PROF_T0()
+                if (active) {
+#pragma unroll 1
+                    for (int j = d - 1; j >= 0; --j) {
+                        const int aj = anc(j);
+                        float acc = is_k ? (j == d - 1 ? 1.f : 0.f) : G[aj * kRows + grow];
+                        if (!p.no_erase) {
+#pragma unroll 1
+                            for (int m = j + 1; m < d; ++m) {
+                                const int am = anc(m);
+                                acc = fmaf(-cf[m] * beta_s[am], G[aj * kRows + am], acc);
+                            }
+                        }
+                        cf[j] = acc;
+                    }
+                }
+                PROF_ADD(7)
+            }
+            // record and M row of operand row `node`: query-row threads on the o walk, key-row threads on the u
+            // walk.  The previous unit's effective vectors must have been formed, its value term issued.
+            if (!(ok = WAIT(3, bar(kRecFree), (useq & 1) ^ 1))) break;
+            if (!(ok = WAIT(5, bar(kMFree), (useq & 1) ^ 1))) break;
+            const bool mine = in_rows && (x.kind == 0 ? !is_k : is_k);
+            if (mine) {
+                uint8_t *rr = rec + node * kRecBytes;
+                uint8_t *mrow = smem + LY::OffM + (node >> 3) * 1024 + (node & 7) * 128;
+#pragma unroll
+                for (int pc = 0; pc < 3; ++pc)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        *reinterpret_cast<uint4 *>(mrow + pc * LY::MPIECE + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+                int cnt = 0;
+                if (active) {
+                    float gamma = 1.f;
+#pragma unroll 1
+                    for (int j = 0; j < d; ++j) gamma *= alpha_s[anc(j)];
+                    const float front = x.kind == 0 ? p.scale : 1.f;
+                    float rho = 1.f;
+#pragma unroll 1
+                    for (int j = d - 1; j >= 0; --j) {
+                        const int a = anc(j);
+                        const float cb = cf[j] * beta_s[a];
+                        // weight of k_a in the effective vector (zero without the erase term) ...
+                        *reinterpret_cast<float *>(rr + kRecW + 4 * j) = p.no_erase ? 0.f : -front * gamma * cb;
+                        *reinterpret_cast<unsigned short *>(rr + kRecOff + 2 * j) =
+                            (unsigned short)((a >> 3) * 1024 + (a & 7) * 128);
+                        // ... and of v_a in the value term, split into three bf16 pieces
+                        float mv = front * rho * cb;
+                        const uint32_t moff = uint32_t((((a >> 3) ^ (node & 7)) << 4) + (a & 7) * 2);
+#pragma unroll
+                        for (int pc = 0; pc < 3; ++pc) {
+                            const __nv_bfloat16 bq = __float2bfloat16_rn(mv);
+                            *reinterpret_cast<__nv_bfloat16 *>(mrow + pc * LY::MPIECE + moff) = bq;
+                            mv -= __bfloat162float(bq);
+                        }
+                        rho *= alpha_s[a];
+                    }
+                    cnt = d;
+                    if (x.kind == 0) {                           // the node's own query row
+                        const int sr = R + node;
+                        *reinterpret_cast<float *>(rr + kRecW + 4 * d) = p.scale * gamma;
+                        *reinterpret_cast<unsigned short *>(rr + kRecOff + 2 * d) =
+                            (unsigned short)((sr >> 3) * 1024 + (sr & 7) * 128);
+                        cnt = d + 1;
+                    }
+                }
+                *reinterpret_cast<int *>(rr) = cnt;
+            }
+            fence_proxy_async();
+            warp_arrive(bar(kMReady), lane);
+            warp_arrive(bar(kRecReady), lane);
+            if (!(ok = solve_sync())) break;                     // nobody reads the Gram block any more
+            if (stid == 0) {
+                // value rows of this unit, as two 64-value blocks per tile, over the scratch
+                const int m = (R >> 4) - 1;
+                const int z = x.l * p.T + x.base;
+                fence_proxy_async();
+                mbar_arrive_expect_tx(bar(kVFull), uint32_t(TP * 2 * R * 128));
+#pragma unroll
+                for (int t = 0; t < TP; ++t)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+                        tma_load_3d(sbase + LY::OffV + (t * 2 + j) * LY::VBLK, &maps.v[m], t * kRows + j * 64, x.h, z,
+                                    bar(kVFull));
             }
             x = nx;
             have = have_next;
             ++useq;
         }
-        if (ok && pend) flush_pend();
-        // everything this warp issued must have completed before TMEM is released
-        if (lane == 0) mma_commit(bar(kDrain));
-        __syncwarp();
-        mbar_wait(bar(kDrain), 0, abort_flag);
+        PROF_STORE()
     } else if (warp < 10) {
-        // ------------------------------------------------------------- preparation
-        const int ptid = threadIdx.x - 64;                       // 0..255
-        const bool solver = warp < 6;                            // these four warps cover the 128 Gram rows
-        const int grow = 32 * (warp & 3) + lane;                 // Gram row (= TMEM lane) of a solver thread
-        const uint32_t lane_addr = uint32_t(32 * (warp & 3)) << 16;
-        const int crow = ptid >> 2, cg = ptid & 3;               // operand row and 8-column group of the slice loop
-        float *scratch = reinterpret_cast<float *>(smem + LY::OffRec);
-        float *Xs = reinterpret_cast<float *>(smem + LY::OffRec);
-        uint8_t *rec = smem + LY::OffRec;
-        float *alpha_s = reinterpret_cast<float *>(smem + LY::OffAlpha);
-        float *beta_s = alpha_s + 64;
-        uint32_t psync = 0, ssync = 0, useq = 0, cc = 0;
-        auto prep_sync = [&]() -> bool {
-            mbar_arrive(bar(kPrepSync));
-            const bool r = wait_fast(bar(kPrepSync), psync & 1, abort_flag);
-            ++psync;
-            return r;
-        };
-        auto solve_sync = [&]() -> bool {
-            mbar_arrive(bar(kSolveSync));
-            const bool r = wait_fast(bar(kSolveSync), ssync & 1, abort_flag);
-            ++ssync;
-            return r;
-        };
+        // ------------------------------------------------------------- effective vectors, one K-slice at a time
+        const int vtid = threadIdx.x - 192;                      // 0..127
+        const int cg = vtid & 3;                                 // 8-column group of the slice
+        const uint8_t *rec = smem + LY::OffRec;
+        uint32_t useq = 0, cc = 0, vsync = 0;
+        PROF_DECL
         auto load_kq = [&](const VUnit &y, int par) {           // one thread
             const int m = (y.npad >> 4) - 1;
             const int z = y.l * p.T + y.base;
@@ -414,272 +639,88 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                 tma_load_3d(stage + c * SCB + y.npad * 128, &maps.q[m], c * 64, y.h, z, bar(kKQFull + par));
             }
         };
-        // per-thread topology and gates of a unit, fetched one unit ahead
-        int4 meta_n = make_int4(0, 0, 0, 0);
-        int meta2_n = 0;
-        float alpha_n = 0.f, beta_n = 0.f;
-        auto fetch_topo = [&](const VUnit &y) {
-            if (solver) {
-                const int node = grow < y.npad ? grow : grow - y.npad;
-                const bool act = grow < 2 * y.npad && node < y.n;
-                meta_n = act ? __ldg(reinterpret_cast<const int4 *>(p.ws.anc) + y.base + node) : make_int4(0, 0, 0, 0);
-                meta2_n = act ? __ldg(p.ws.anc2 + 4 * (y.base + node)) : 0;
-            }
-            if (ptid < y.n) {
-                const int r = (y.l * p.T + y.base + ptid) * p.H + y.h;
-                alpha_n = __ldg(p.alpha + r);
-                beta_n = __ldg(p.beta + r);
-            }
-        };
-
         VUnit x, nx, nx2;
         bool ok = true;
         bool have = first_unit(walk, x);
-        if (have) {
+        if (have && vtid == 0) {
             nx = x;
-            const bool h2 = next_unit(walk, nx);
-            if (ptid == 0) {
-                load_kq(x, 0);
-                if (h2) load_kq(nx, 1);
-            }
-            fetch_topo(x);
+            load_kq(x, 0);
+            if (next_unit(walk, nx)) load_kq(nx, 1);
         }
         while (have && ok) {
             const int par = useq & 1;
             const int R = x.npad;
-            const int4 meta = meta_n;
-            const int meta2 = meta2_n;
             nx = x;
             const bool have_next = next_unit(walk, nx);
             nx2 = nx;
             const bool have_next2 = have_next && next_unit(walk, nx2);
-            // value rows of this unit (the buffer is free once the previous unit's value term has been read)
-            if (warp == 2) {
-                if (!(ok = wait_fast(bar(kVFree), (useq & 1) ^ 1, abort_flag))) break;
-                if (lane == 0) {
-                    const int m = (R >> 4) - 1;
-                    const int z = x.l * p.T + x.base;
-                    mbar_arrive_expect_tx(bar(kVFull), uint32_t(TP * 2 * R * 128));
-#pragma unroll
-                    for (int t = 0; t < TP; ++t)
-#pragma unroll
-                        for (int j = 0; j < 2; ++j)
-                            tma_load_3d(sbase + LY::OffV + (t * 2 + j) * LY::VBLK, &maps.v[m], t * kRows + j * 64, x.h, z,
-                                        bar(kVFull));
-                }
-                __syncwarp();
-            }
-            if (ptid < x.n) { alpha_s[ptid] = alpha_n; beta_s[ptid] = beta_n; }
-            if (have_next) fetch_topo(nx);
-            if (!(ok = wait_fast(bar(kKQFull + par), (useq >> 1) & 1, abort_flag))) break;
-            if (!(ok = wait_fast(bar(kGramFull), useq & 1, abort_flag))) break;
-            tc_fence_after();
-
-            // this thread's Gram row belongs to node `node` (key rows first, then query rows)
-            const bool is_k = grow < R;
-            const int node = is_k ? grow : grow - R;
-            const bool in_rows = solver && grow < 2 * R;
-            const bool active = in_rows && node < x.n;
-            const int d = active ? (meta.x & 0xff) : 0;
-            const int ng = is_k ? d - 1 : d;                      // Gram entries this row needs: ancestors (+ itself)
-            float g[kMaxD];
-#pragma unroll
-            for (int j = 0; j < kMaxD; ++j) g[j] = 0.f;
-            if (solver) {
-                const uint32_t gaddr = tmem_base + par * kPairCols + lane_addr;
+            if (!(ok = WAIT(3, bar(kKQFull + par), (useq >> 1) & 1))) break;
+            if (!(ok = WAIT(4, bar(kRecReady), useq & 1))) break;
+            const uint8_t *stage = smem + LY::OffStage + par * LY::STAGE;
+            for (int c = 0; c < NC; ++c, ++cc) {
+                const int bb = cc & 1;
+                if (!(ok = WAIT(6, bar(kBFree + bb), ((cc >> 1) & 1) ^ 1))) break;
+                PROF_T0()
+                const uint8_t *region = stage + (c >> 1) * SCB;
+                const uint32_t slot = uint32_t((c & 1) * 4 + cg);
+                uint8_t *bbuf = smem + LY::OffB + bb * LY::BBUF;
 #pragma unroll 1
-                for (int c0 = 0; c0 < R; c0 += 8) {
-                    float t8[8];
-                    tmem_ld8(gaddr + c0, t8);
-                    tmem_ld_wait();
+                for (int crow = vtid >> 2; crow < R; crow += 32) {
+                    const uint8_t *rr = rec + crow * kRecBytes;
+                    const int cnt = *reinterpret_cast<const int *>(rr);
+                    float acc[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) scratch[i * kRows + grow] = t8[i];
-#pragma unroll
-                    for (int j = 0; j < kMaxD; ++j) {
-                        const int a = j < d - 1 ? anc_at(meta, meta2, j) : node;
-                        if (j < ng && (a >> 3) == (c0 >> 3)) g[j] = scratch[(a & 7) * kRows + grow];
+                    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll 2
+                    for (int j = 0; j < cnt; ++j) {
+                        const float w = *reinterpret_cast<const float *>(rr + kRecW + 4 * j);
+                        const uint32_t off = *reinterpret_cast<const unsigned short *>(rr + kRecOff + 2 * j);
+                        const uint4 raw = *reinterpret_cast<const uint4 *>(region + off + ((slot ^ ((off >> 7) & 7u)) << 4));
+                        acc[0] = fmaf(w, bf_lo(raw.x), acc[0]); acc[1] = fmaf(w, bf_hi(raw.x), acc[1]);
+                        acc[2] = fmaf(w, bf_lo(raw.y), acc[2]); acc[3] = fmaf(w, bf_hi(raw.y), acc[3]);
+                        acc[4] = fmaf(w, bf_lo(raw.z), acc[4]); acc[5] = fmaf(w, bf_hi(raw.z), acc[5]);
+                        acc[6] = fmaf(w, bf_lo(raw.w), acc[6]); acc[7] = fmaf(w, bf_hi(raw.w), acc[7]);
                     }
-                }
-                tc_fence_before();
-                mbar_arrive(bar(kGramDone));                     // the state MMAs may now overwrite these columns
-            }
-            if (!(ok = prep_sync())) break;                      // gates visible; Gram scratch dead
-
-            // X rows (gate-free (I + Ahat)^-1 along the path), level by level
-            float xr[kMaxD];
+                    float hi[8], lo[8];
 #pragma unroll
-            for (int j = 0; j < kMaxD; ++j) xr[j] = 0.f;
-            const float my_beta = active ? beta_s[node] : 0.f;
-            if (solver) {
-                if (!p.no_erase) {
-                    for (int lev = 2; lev <= p.max_depth && ok; ++lev) {
-                        if (active && is_k && d == lev) {
-#pragma unroll
-                            for (int j = 0; j < kMaxD - 1; ++j) {
-                                if (j < d - 1) {
-                                    float acc = 0.f;
-#pragma unroll
-                                    for (int m = j; m < kMaxD - 1; ++m) {
-                                        if (m < d - 1) {
-                                            const float xv = (m == j) ? 1.f : Xs[anc_at(meta, meta2, m) * kMaxD + j];
-                                            acc = fmaf(g[m], xv, acc);
-                                        }
-                                    }
-                                    xr[j] = -my_beta * acc;
-                                    Xs[node * kMaxD + j] = xr[j];
-                                }
-                            }
-                        }
-                        ok = solve_sync();
-                    }
-                    if (!ok) break;
-                }
-                // query rows: C = Phat X over the path (entry d-1 pairs with the node's own key)
-                if (active && !is_k) {
-#pragma unroll
-                    for (int j = 0; j < kMaxD; ++j) {
-                        if (j < d) {
-                            float acc = 0.f;
-                            if (p.no_erase) {
-                                acc = g[j];
-                            } else {
-#pragma unroll
-                                for (int m = j; m < kMaxD; ++m) {
-                                    if (m < d) {
-                                        const int am = m < d - 1 ? anc_at(meta, meta2, m) : node;
-                                        const float xv = (m == j) ? 1.f : Xs[am * kMaxD + j];
-                                        acc = fmaf(g[m], xv, acc);
-                                    }
-                                }
-                            }
-                            xr[j] = acc;
-                        }
-                    }
-                } else if (active && is_k) {
-#pragma unroll
-                    for (int j = 0; j < kMaxD; ++j)
-                        if (j == d - 1) xr[j] = 1.f;
-                }
-                if (!(ok = solve_sync())) break;                 // X rows dead: the records may take their place
-
-                // record and M row of operand row `node`: query-row threads on the o walk, key-row threads on the u walk
-                const bool mine = in_rows && (x.kind == 0 ? !is_k : is_k);
-                // the previous unit's value term must have read the pieces of M
-                if (!(ok = wait_fast(bar(kMFree), (useq & 1) ^ 1, abort_flag))) break;
-                if (mine) {
-                    uint8_t *rr = rec + node * kRecBytes;
-                    uint8_t *mrow = smem + LY::OffM + (node >> 3) * 1024 + (node & 7) * 128;
-#pragma unroll
-                    for (int pc = 0; pc < 3; ++pc)
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            *reinterpret_cast<uint4 *>(mrow + pc * LY::MPIECE + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-                    int cnt = 0;
-                    if (active) {
-                        float gamma = 1.f;
-#pragma unroll
-                        for (int j = 0; j < kMaxD; ++j)
-                            if (j < d) gamma *= alpha_s[j < d - 1 ? anc_at(meta, meta2, j) : node];
-                        const float front = x.kind == 0 ? p.scale : 1.f;
-                        float rho = 1.f;
-#pragma unroll
-                        for (int j = kMaxD - 1; j >= 0; --j) {
-                            if (j < d) {
-                                const int a = j < d - 1 ? anc_at(meta, meta2, j) : node;
-                                const float cb = xr[j] * beta_s[a];
-                                // weight of k_a in the effective vector (zero without the erase term) ...
-                                const float w = p.no_erase ? 0.f : -front * gamma * cb;
-                                *reinterpret_cast<float *>(rr + kRecW + 4 * j) = w;
-                                *reinterpret_cast<unsigned short *>(rr + kRecOff + 2 * j) =
-                                    (unsigned short)((a >> 3) * 1024 + (a & 7) * 128);
-                                // ... and of v_a in the value term, split into three bf16 pieces
-                                float mv = front * rho * cb;
-                                if (p.no_erase && x.kind == 1) mv = (j == d - 1) ? beta_s[a] : 0.f;
-                                const uint32_t moff = uint32_t((((a >> 3) ^ (node & 7)) << 4) + (a & 7) * 2);
-#pragma unroll
-                                for (int pc = 0; pc < 3; ++pc) {
-                                    const __nv_bfloat16 b = __float2bfloat16_rn(mv);
-                                    *reinterpret_cast<__nv_bfloat16 *>(mrow + pc * LY::MPIECE + moff) = b;
-                                    mv -= __bfloat162float(b);
-                                }
-                                rho *= alpha_s[a];
-                            }
-                        }
-                        cnt = d;
-                        if (x.kind == 0) {                       // the node's own query row
-                            const int sr = R + node;
-                            *reinterpret_cast<float *>(rr + kRecW + 4 * d) = p.scale * gamma;
-                            *reinterpret_cast<unsigned short *>(rr + kRecOff + 2 * d) =
-                                (unsigned short)((sr >> 3) * 1024 + (sr & 7) * 128);
-                            cnt = d + 1;
-                        }
-                    }
-                    *reinterpret_cast<int *>(rr) = cnt;
+                    for (int i = 0; i < 8; ++i) { hi[i] = round_tf32(acc[i]); lo[i] = acc[i] - hi[i]; }
+                    const int r0 = crow, r1 = R + crow;
+                    uint8_t *d0 = bbuf + (r0 >> 3) * 1024 + (r0 & 7) * 128;
+                    uint8_t *d1 = bbuf + (r1 >> 3) * 1024 + (r1 & 7) * 128;
+                    *reinterpret_cast<float4 *>(d0 + (((2 * cg) ^ (r0 & 7)) << 4)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<float4 *>(d0 + (((2 * cg + 1) ^ (r0 & 7)) << 4)) = make_float4(hi[4], hi[5], hi[6], hi[7]);
+                    *reinterpret_cast<float4 *>(d1 + (((2 * cg) ^ (r1 & 7)) << 4)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                    *reinterpret_cast<float4 *>(d1 + (((2 * cg + 1) ^ (r1 & 7)) << 4)) = make_float4(lo[4], lo[5], lo[6], lo[7]);
                 }
                 fence_proxy_async();
-                mbar_arrive(bar(kMReady));
+                warp_arrive(bar(kBReady + bb), lane);
+                PROF_ADD(7)
             }
-            if (!(ok = prep_sync())) break;                      // records visible
-
-            // effective vectors, one K-slice (32 columns) at a time: this thread's row, 8 columns
-            {
-                const bool on = crow < R;
-                const uint8_t *rr = rec + crow * kRecBytes;
-                const int cnt = on ? *reinterpret_cast<const int *>(rr) : 0;
-                const uint8_t *stage = smem + LY::OffStage + par * LY::STAGE;
-                for (int c = 0; c < NC; ++c, ++cc) {
-                    const int bb = cc & 1;
-                    if (!(ok = wait_fast(bar(kBFree + bb), ((cc >> 1) & 1) ^ 1, abort_flag))) break;
-                    if (on) {
-                        float acc[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-                        const uint8_t *region = stage + (c >> 1) * SCB;
-                        const uint32_t slot = uint32_t((c & 1) * 4 + cg);
-                        for (int j = 0; j < cnt; ++j) {
-                            const float w = *reinterpret_cast<const float *>(rr + kRecW + 4 * j);
-                            const uint32_t off = *reinterpret_cast<const unsigned short *>(rr + kRecOff + 2 * j);
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(region + off + ((slot ^ ((off >> 7) & 7u)) << 4));
-                            acc[0] = fmaf(w, bf_lo(raw.x), acc[0]); acc[1] = fmaf(w, bf_hi(raw.x), acc[1]);
-                            acc[2] = fmaf(w, bf_lo(raw.y), acc[2]); acc[3] = fmaf(w, bf_hi(raw.y), acc[3]);
-                            acc[4] = fmaf(w, bf_lo(raw.z), acc[4]); acc[5] = fmaf(w, bf_hi(raw.z), acc[5]);
-                            acc[6] = fmaf(w, bf_lo(raw.w), acc[6]); acc[7] = fmaf(w, bf_hi(raw.w), acc[7]);
-                        }
-                        float hi[8], lo[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) { hi[i] = round_tf32(acc[i]); lo[i] = acc[i] - hi[i]; }
-                        uint8_t *bbuf = smem + LY::OffB + bb * LY::BBUF;
-                        const int r0 = crow, r1 = R + crow;
-                        uint8_t *d0 = bbuf + (r0 >> 3) * 1024 + (r0 & 7) * 128;
-                        uint8_t *d1 = bbuf + (r1 >> 3) * 1024 + (r1 & 7) * 128;
-                        *reinterpret_cast<float4 *>(d0 + (((2 * cg) ^ (r0 & 7)) << 4)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                        *reinterpret_cast<float4 *>(d0 + (((2 * cg + 1) ^ (r0 & 7)) << 4)) = make_float4(hi[4], hi[5], hi[6], hi[7]);
-                        *reinterpret_cast<float4 *>(d1 + (((2 * cg) ^ (r1 & 7)) << 4)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
-                        *reinterpret_cast<float4 *>(d1 + (((2 * cg + 1) ^ (r1 & 7)) << 4)) = make_float4(lo[4], lo[5], lo[6], lo[7]);
-                    }
-                    fence_proxy_async();
-                    mbar_arrive(bar(kBReady + bb));
-                }
-                if (!ok) break;
-            }
-            if (!(ok = prep_sync())) break;                      // staged rows and records of this unit are dead
-            if (ptid == 0 && have_next2) load_kq(nx2, par);
+            if (!ok) break;
+            warp_arrive(bar(kRecFree), lane);                    // the records of this unit are dead
+            // every warp of the role has left the staged rows of this unit: request those of the unit after next
+            warp_arrive(bar(kVecSync), lane);
+            if (!(ok = WAIT(0, bar(kVecSync), vsync & 1))) break;
+            ++vsync;
+            if (vtid == 0 && have_next2) load_kq(nx2, par);
             x = nx;
             have = have_next;
             ++useq;
         }
+        PROF_STORE()
     } else if (warp < 14) {
         // ------------------------------------------------------------- TF32 remainder of every slice, in place
         const int stid = threadIdx.x - 10 * 32;
         uint32_t it = 0;
         VUnit x;
         bool ok = true;
+        PROF_DECL
         for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
             for (int i = 0; i < TP * NC; ++i, ++it) {
                 const int s = it % NS;
                 const uint32_t ph = (it / NS) & 1;
-                if (!(ok = wait_fast(bar(kFull + s), ph, abort_flag))) break;
-                if (!(ok = wait_fast(bar(kP1Done + s), ph, abort_flag))) break;
+                if (!(ok = WAIT(0, bar(kFull + s), ph))) break;
+                if (!(ok = WAIT(1, bar(kP1Done + s), ph))) break;
                 float4 *sl = reinterpret_cast<float4 *>(smem + LY::OffRing + s * kSliceBytes);
 #pragma unroll
                 for (int k = 0; k < kSliceBytes / 16 / kSplitThreads; ++k) {
@@ -691,9 +732,10 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                     sl[stid + k * kSplitThreads] = v;
                 }
                 fence_proxy_async();
-                mbar_arrive(bar(kLo + s));
+                warp_arrive(bar(kLo + s), lane);
             }
         }
+        PROF_STORE()
     } else {
         // ------------------------------------------------------------- epilogue
         const int row = 32 * (warp & 3) + lane;
@@ -701,9 +743,10 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
         uint32_t useq = 0;
         VUnit x;
         bool ok = true;
+        PROF_DECL
         for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x), ++useq) {
             const int pr = useq & 1;
-            if (!(ok = wait_fast(bar(kAccFull + pr), (useq >> 1) & 1, abort_flag))) break;
+            if (!(ok = WAIT(0, bar(kAccFull + pr), (useq >> 1) & 1))) break;
             tc_fence_after();
             const int R = x.npad, n = x.n;
             const size_t rec0 = size_t((x.l * p.T + x.base) * p.H + x.h);
@@ -724,8 +767,9 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                 }
             }
             tc_fence_before();
-            mbar_arrive(bar(kPairFree + pr));
+            warp_arrive(bar(kPairFree + pr), lane);
         }
+        PROF_STORE()
     }
 
     tc_fence_before();

@@ -145,7 +145,6 @@ static_assert(kBarCount <= 40, "barrier region too small");
         for (int i_ = 0; i_ < 8; ++i_) dst[i_] = prof_w[i_];                                      \
         dst[8] = clock64() - prof_t0;                                                             \
     }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag);
 __device__ __forceinline__ bool prof_wait(long long &acc, uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
     const long long t = clock64();
