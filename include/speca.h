@@ -87,6 +87,7 @@ extern "C" {
 #define SPECA_ROUTE_SERIAL      1   /* state-resident walk, one rank-1 update per node (Section 4.1) */
 #define SPECA_ROUTE_FACTORIZED  2   /* tree-masked factorised form on tensor cores (Section 4.2), fp32-grade */
 #define SPECA_ROUTE_TF32        3   /* the same factorisation with the state read once as TF32 (single pass)  */
+#define SPECA_ROUTE_EFFECTIVE   4   /* effective-query form of the factorisation, fp32-grade (trees up to 16 levels) */
 /* SPECA_ROUTE_FACTORIZED takes d_v in {128, 256}, max_depth <= 16 and max_nodes <= 64 (d_k = 128) or <= 32
  * (d_k = 256).  Both tensor-core operands are split into a TF32 head and its exact remainder, so outputs
  * carry fp32 accuracy whatever the magnitude of the state.  AUTO uses it whenever it applies and the serial

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libspeca.so")
 OK = 0
 STATUS_BAD_PARENT, STATUS_BAD_OFFSETS, STATUS_BAD_PATH, STATUS_TOO_DEEP = 1, 2, 4, 8
 STATUS_TOO_MANY, STATUS_TIMEOUT, STATUS_BAD_DEPTH = 16, 32, 64
-ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED = 0, 1, 2
+ROUTE_AUTO, ROUTE_SERIAL, ROUTE_FACTORIZED, ROUTE_TF32, ROUTE_EFFECTIVE = 0, 1, 2, 3, 4
 RULE_GATED_DELTA, RULE_GATED_NO_ERASE = 0, 1
 
 EXPORTS = ["speca_version", "speca_strerror", "speca_workspace_bytes", "speca_decode_step",

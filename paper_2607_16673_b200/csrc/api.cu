@@ -15,7 +15,7 @@ int check_dims(const speca_dims *d)
     if (d->d_v < 32 || d->d_v > 1024 || d->d_v % 32 != 0) return SPECA_ERR_UNSUPPORTED;
     if (d->max_depth < 1 || d->max_depth > 16) return SPECA_ERR_RANGE;
     if (d->max_nodes < 1 || d->max_nodes > 1024) return SPECA_ERR_RANGE;
-    if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_TF32) return SPECA_ERR_UNSUPPORTED;
+    if (d->route < SPECA_ROUTE_AUTO || d->route > SPECA_ROUTE_EFFECTIVE) return SPECA_ERR_UNSUPPORTED;
     if (d->rule != SPECA_RULE_GATED_DELTA && d->rule != SPECA_RULE_GATED_NO_ERASE) return SPECA_ERR_UNSUPPORTED;
     const long long units = 1LL * d->n_layers * d->batch * d->heads;
     if (units * (d->d_v / 2) > 0x7fffffffLL) return SPECA_ERR_RANGE;       // grid size bound
@@ -65,20 +65,24 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
     p.status = status_word;
     p.ws = carve_workspace(workspace, dims->batch, total_nodes);
     p.n_slots = tree_slots_needed(dims->max_nodes);
-    // AUTO: the fp32-grade tensor-core route where the shape fits, else the serial walk.  The single-pass
-    // TF32 kernel runs only when asked for by name.
+    // AUTO: an fp32-grade tensor-core route where the shape fits -- the factorised kernel in its compensated form,
+    // or, for shapes it does not take (more than 32 nodes below 16 levels), the effective-query kernel -- else the
+    // serial walk.  The single-pass TF32 kernel runs only when asked for by name.
     const bool tf32 = dims->route == SPECA_ROUTE_TF32;
     if (tf32 && !factorized_supported(dims)) return SPECA_ERR_UNSUPPORTED;
-    const bool can_eff = effective_supported(dims);
-    if (dims->route == SPECA_ROUTE_FACTORIZED && !can_eff) return SPECA_ERR_UNSUPPORTED;
-    const bool eff = can_eff && (dims->route == SPECA_ROUTE_AUTO || dims->route == SPECA_ROUTE_FACTORIZED);
-    if (!chain || eff || tf32) {
+    const bool tensor = dims->route == SPECA_ROUTE_AUTO || dims->route == SPECA_ROUTE_FACTORIZED;
+    const bool fact = tensor && factorized_supported(dims);
+    if (dims->route == SPECA_ROUTE_EFFECTIVE && !effective_supported(dims)) return SPECA_ERR_UNSUPPORTED;
+    const bool eff = dims->route == SPECA_ROUTE_EFFECTIVE || (tensor && !fact && effective_supported(dims));
+    if (dims->route == SPECA_ROUTE_FACTORIZED && !fact && !eff) return SPECA_ERR_UNSUPPORTED;
+    if (!chain || fact || eff || tf32) {
         // with parent == NULL (chain entry point) the plan kernel assumes parent[i] = i - 1
         rc = cuda_rc(launch_plan(p, st));
         if (rc != SPECA_OK) return rc;
     }
+    if (fact) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, true, st));
     if (eff) return cuda_rc(launch_verify_effective(p, dims->d_k, st));
-    if (tf32) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, st));
+    if (tf32) return cuda_rc(launch_verify_factorized(p, dims->d_k, false, false, st));
     return cuda_rc(launch_verify_serial(p, dims->d_k, chain, st));
 }
 
@@ -110,6 +114,15 @@ void *noalloc_scratch_for_current_device()
 extern "C" {
 
 int speca_version(void) { return SPECA_VERSION; }
+
+/* Test hook, deliberately absent from speca.h: makes the next tensor-core verifications withhold the first
+ * state slice of CTA 0, so that its bounded waits expire and the call reports SPECA_STATUS_TIMEOUT without
+ * faulting anything.  The failure-detection test switches it on for one call and off again. */
+void speca_test_withhold_first_load(int on)
+{
+    factorized_set_withhold(on);
+    effective_set_withhold(on);
+}
 
 const char *speca_strerror(int code)
 {
@@ -350,7 +363,7 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S, const uint16_t *k
     if (rc != SPECA_OK) return rc;
     rc = cuda_rc(launch_pending_check(p, 8, st));
     if (rc != SPECA_OK) return rc;
-    return cuda_rc(launch_verify_factorized(p, dims->d_k, true, st));
+    return cuda_rc(launch_verify_factorized(p, dims->d_k, true, false, st));
 }
 
 }  // extern "C"

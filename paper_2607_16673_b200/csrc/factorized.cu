@@ -75,6 +75,7 @@ constexpr int kThreads = 14 * 32;
 constexpr int kUpdWarps = 2;                   // state-update role of the fused kernel
 constexpr int kUpdThreads = kUpdWarps * 32;
 constexpr int kThreadsFused = kThreads + kUpdThreads;
+constexpr int kThreadsComp = kThreads + 5 * 32;  // compensated form: a second MMA issuer and four warps that rewrite slices
 constexpr int kPrepThreads = 128;
 // The tensor core reads an fp32 state element as TF32 by dropping its low 13 mantissa bits, i.e. it
 // rounds every element toward zero: on average a value with mantissa m in [1, 2) loses 2^-11 / m of
@@ -96,7 +97,7 @@ constexpr int kOffGram = kOffStage + 2 * kStageChunkBytes;
 constexpr int kOffCoef = kOffGram + kGramHalf * kTileRows * 4;
 constexpr int kOffAlpha = kOffCoef + 2 * kMaxNodes * kCoefStride * 4;
 constexpr int kOffBars = kOffAlpha + 2 * kMaxNodes * 4;                   // alpha, beta by position
-constexpr int kOffMisc = kOffBars + 8 * 40;
+constexpr int kOffMisc = kOffBars + 8 * 56;
 constexpr int kOffPendK = kOffMisc + 64;                                  // bf16 keys of the pending path [2][8][d_k + 8]
 constexpr int kKeyStride = kDK * 2 + 16;                                   // bytes per staged pending key (bank padding)
 constexpr int kKeyBuf = kMaxDepth * kKeyStride;
@@ -128,9 +129,11 @@ enum Bar {
     kBarUpd,                             // [kStages] fused only: update role -> MMA, slice advanced in place
     kBarPendFull = kBarUpd + kStages,    // [2] fused only: TMA producer -> update role, pending u rows and keys staged
     kBarPendFree = kBarPendFull + 2,     // [2] fused only: update role -> TMA producer
+    kBarP1Done = kBarPendFree + 2,       // [kStages] compensated form: MMA -> split warps, first pass has read the slice
+    kBarLo = kBarP1Done + kStages,       // [kStages] compensated form: split warps -> MMA, slice rewritten as its remainder
     kBarCount
 };
-static_assert(kBarCount <= 40, "barrier region too small");
+static_assert(kBarCount <= 56, "barrier region too small");
 
 
 // Optional self-profiling build (-DSPECA_PROF): cycles spent in each kind of wait per role.
@@ -383,8 +386,12 @@ __device__ __forceinline__ void node_step_deep(float (&ustk)[TP][MAXD], const fl
 // DK = key width, 128 or 256.  The operand buffers have a fixed size, so the wider key halves
 // the number of [K;Q] rows they hold: up to 64 nodes per sequence at d_k = 128, 32 at d_k = 256.
 // DEEP: trees up to 16 levels deep (up to 32 nodes per sequence at either key width; not with FUSED).
-template <int TP, bool FUSED, int DK = kDK, bool DEEP = false>
-__global__ void __launch_bounds__(FUSED ? kThreadsFused : kThreads, 1)
+// COMP: compensated form (not with FUSED).  The tensor core reads the fp32 state as TF32, i.e. its top 19 bits;
+// every slice is therefore multiplied twice: as landed, and, rewritten in place as its exact remainder
+// S - tf32(S) by two extra warps, once more into the same accumulator.  [K;Q] is exact in TF32, so R and G carry
+// fp32 accuracy (the dropped part is 2^-21 of the state).  The two value tiles are then issued by two warps.
+template <int TP, bool FUSED, int DK = kDK, bool DEEP = false, bool COMP = false>
+__global__ void __launch_bounds__(FUSED ? kThreadsFused : (COMP ? kThreadsComp : kThreads), 1)
 verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid_constant__ KQMaps kq, FParams fp)
 {
     // The swizzled operand regions need 1024-byte alignment.  The array is declared with that
@@ -410,20 +417,22 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             mbar_init(bar(kBarFull + s), 1);
             mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarUpd + s), kUpdThreads);
+            mbar_init(bar(kBarP1Done + s), 1);
+            mbar_init(bar(kBarLo + s), 4);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarPendFull + i), 1); mbar_init(bar(kBarPendFree + i), kUpdThreads); }
         mbar_init(bar(kBarBReady), kPrepThreads);
-        mbar_init(bar(kBarBFree), 1);
+        mbar_init(bar(kBarBFree), COMP ? TP : 1);
         mbar_init(bar(kBarStageReady), 1);
         mbar_init(bar(kBarGramFull), 1);
         mbar_init(bar(kBarGramDone), kPrepThreads);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kBarCoefReady + i), kPrepThreads);
             mbar_init(bar(kBarCoefFree + i), 128);
-            mbar_init(bar(kBarAccFull + i), 1);
+            mbar_init(bar(kBarAccFull + i), COMP ? TP : 1);
             mbar_init(bar(kBarPairFree + i), 128);
         }
-        mbar_init(bar(kBarDrain), 1);
+        mbar_init(bar(kBarDrain), COMP ? TP : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int b = threadIdx.x; b < p.B && b < kWalkSeqs; b += blockDim.x) {
@@ -454,6 +463,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     constexpr int SCB = BROWS * 128;                              // bytes of one such chunk
     static_assert(NC * BCB == kChunks * kBopChunkBytes && SC * SCB == 2 * kStageChunkBytes, "operand buffers keep their size");
     static_assert(!(FUSED && DEEP), "the fused kernel takes pending paths and trees of at most 8 levels");
+    static_assert(!(FUSED && COMP), "the fused kernel reads the state in a single TF32 pass");
     constexpr int MAXD = DEEP ? 2 * kMaxDepth : kMaxDepth;        // tree depth this instantiation takes
     constexpr int CS = 2 * MAXD + 4;                              // floats of a coefficient record
     constexpr int MAXN = DEEP ? kMaxNodes / 2 : BROWS / 2;        // nodes per sequence; also the stride of the coefficient buffers
@@ -604,11 +614,14 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             // the value rows of this unit's nodes are read by the epilogue with plain loads a
             // couple of units from now: pull them into L2 meanwhile
             if (lane == 0 && x.n > 0) tma_prefetch_3d(&kq.v[(x.npad >> 4) - 1], 0, x.h, x.l * p.T + x.base);
-            for (int t = 0; t < TP && ok; ++t) {
-                // tile t of a unit holds its value rows t, t + TP, t + 2 TP, ... (interleaved tiles:
-                // an epilogue thread then owns TP ADJACENT value rows, one per tile)
-                const int row = x.u * kTileRows;                      // row-group in the [units*128][TP][d_k] view of S0
-                for (int c = 0; c < NC; ++c, ++it) {
+            // tile t of a unit holds its value rows t, t + TP, t + 2 TP, ... (interleaved tiles:
+            // an epilogue thread then owns TP ADJACENT value rows, one per tile).  Slices go tile by tile,
+            // or, in the compensated form (one MMA issuer per tile), K-slice by K-slice over both tiles.
+            const int row = x.u * kTileRows;                          // row-group in the [units*128][TP][d_k] view of S0
+            for (int o = 0; o < TP && ok; ++o) {
+                for (int i = 0; i < NC; ++i, ++it) {
+                    const int lin = o * NC + i;
+                    const int t = COMP ? lin % TP : o, c = COMP ? lin / TP : i;
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
                     if (!(ok = WAIT(0, bar(kBarEmpty + s), ph ^ 1))) break;
@@ -625,6 +638,132 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         if (*abort_flag) {
             const uint64_t t0 = global_timer_ns();
             while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+        }
+    } else if (COMP && (warp == 1 || warp == 14)) {
+        // ------------------------------------------------------------- MMA issuers of the compensated form
+        // One warp per value tile (disjoint accumulator columns); warp 1 also issues the Gram blocks.  Per slice:
+        // first pass as landed, then -- one slice later, so that the rewrite in between is rarely waited for --
+        // the second pass over the remainder, which releases the slot.
+        const int mt = warp == 1 ? 0 : 1;
+        uint32_t unit_seq = 0;
+        Unit x;
+        bool ok = mt < TP;
+        const uint32_t bop = sbase + kOffBop, stage = sbase + kOffStage;
+        auto issue_gram = [&](uint32_t seq, int npad) -> bool {
+            const int pr = seq & 1;
+            if (!wait_fast(bar(kBarStageReady), seq & 1, abort_flag)) return false;
+            if (!wait_fast(bar(kBarPairFree + pr), ((seq >> 1) & 1) ^ 1, abort_flag)) return false;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t idg = make_idesc_bf16(npad);
+#pragma unroll
+                for (int c = 0; c < SC; ++c)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t d = make_desc(stage + c * SCB + k * 32);
+                        mma_bf16(tmem_base + pr * kPairCols, d, d, idg, (c | k) != 0);
+                    }
+                mma_commit(bar(kBarGramFull));
+            }
+            __syncwarp();
+            return true;
+        };
+        bool have = ok && first_unit(walk, x);
+        if (have && mt == 0) ok = issue_gram(0, x.npad);
+        while (have && ok) {
+            const int pr = unit_seq & 1;
+            const uint32_t acc = tmem_base + pr * kPairCols + mt * kAccCols;
+            if (!(ok = wait_fast(bar(kBarBReady), unit_seq & 1, abort_flag))) break;
+            if (mt == 0) {
+                if (!(ok = wait_fast(bar(kBarGramDone), unit_seq & 1, abort_flag))) break;
+            } else if (!(ok = wait_fast(bar(kBarPairFree + pr), ((unit_seq >> 1) & 1) ^ 1, abort_flag))) {
+                break;
+            }
+            tc_fence_after();
+            const uint32_t idm = make_idesc(2 * x.npad);
+            int ps = -1;
+            uint32_t pph = 0;
+            for (int c = 0; c <= NC && ok; ++c) {
+                if (c < NC) {
+                    const uint32_t it = (unit_seq * NC + c) * TP + mt;
+                    const int s = it % NS;
+                    const uint32_t ph = (it / NS) & 1;
+                    if (!(ok = wait_fast(bar(kBarFull + s), ph, abort_flag))) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t sa = sbase + kOffRing + s * kStageBytes;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_tf32(acc, make_desc(sa + k * 32), make_desc(bop + c * BCB + k * 32), idm, (c | k) != 0);
+                        mma_commit(bar(kBarP1Done + s));
+                    }
+                    __syncwarp();
+                    if (ps >= 0) {
+                        if (!(ok = wait_fast(bar(kBarLo + ps), pph, abort_flag))) break;
+                        tc_fence_after();
+                        if (lane == 0) {
+                            const uint32_t sa = sbase + kOffRing + ps * kStageBytes;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                mma_tf32(acc, make_desc(sa + k * 32), make_desc(bop + (c - 1) * BCB + k * 32), idm, 1);
+                            mma_commit(bar(kBarEmpty + ps));
+                        }
+                        __syncwarp();
+                    }
+                    ps = s; pph = ph;
+                } else {
+                    // the last slice's second pass closes the tile
+                    if (!(ok = wait_fast(bar(kBarLo + ps), pph, abort_flag))) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t sa = sbase + kOffRing + ps * kStageBytes;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_tf32(acc, make_desc(sa + k * 32), make_desc(bop + (NC - 1) * BCB + k * 32), idm, 1);
+                        mma_commit(bar(kBarEmpty + ps));
+                        mma_commit(bar(kBarAccFull + pr));
+                        mma_commit(bar(kBarBFree));
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!ok) break;
+            ++unit_seq;
+            have = next_unit(walk, x);
+            if (have && mt == 0) ok = issue_gram(unit_seq, x.npad);
+        }
+        // everything this warp issued must have completed before TMEM is released
+        if (mt < TP) {
+            if (lane == 0) mma_commit(bar(kBarDrain));
+            __syncwarp();
+            mbar_wait(bar(kBarDrain), 0, abort_flag);
+        }
+    } else if (COMP && warp >= 15) {
+        // ------------------------------------------------------------- compensated form: remainder of every slice, in place
+        const int stid = threadIdx.x - 15 * 32;                  // 0..127
+        uint32_t it = 0;
+        Unit x;
+        bool ok = true;
+        for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
+            for (int i = 0; i < TP * NC; ++i, ++it) {
+                const int s = it % NS;
+                const uint32_t ph = (it / NS) & 1;
+                if (!(ok = wait_fast(bar(kBarFull + s), ph, abort_flag))) break;
+                if (!(ok = wait_fast(bar(kBarP1Done + s), ph, abort_flag))) break;
+                float4 *sl = reinterpret_cast<float4 *>(smem + kOffRing + s * kStageBytes);
+#pragma unroll
+                for (int k = 0; k < kStageBytes / 16 / 128; ++k) {
+                    float4 v = sl[stid + k * 128];
+                    v.x -= __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+                    v.y -= __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+                    v.z -= __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+                    v.w -= __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+                    sl[stid + k * 128] = v;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarLo + s));
+            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
@@ -879,7 +1018,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                     for (int i = 0; i < MAXD / 4; ++i)
                         reinterpret_cast<float4 *>(cf)[i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
-                    cf[2 * MAXD] = (active && !p.no_erase) ? sgn * ratio * kDebias : 0.f;      // cR = -beta gamma
+                    cf[2 * MAXD] = (active && !p.no_erase) ? sgn * ratio * (COMP ? 1.f : kDebias) : 0.f;      // cR = -beta gamma
                 } else {
                     // level d-1 is the node itself: (q_t . k_t) with ratio 1
                     c[MAXD - 1] = 0.f;
@@ -889,7 +1028,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
 #pragma unroll
                     for (int i = 0; i < MAXD / 4; ++i)
                         reinterpret_cast<float4 *>(cf)[MAXD / 4 + i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
-                    cf[2 * MAXD + 1] = active ? sgn * ratio * kDebias : 0.f;                  // cG = scale gamma
+                    cf[2 * MAXD + 1] = active ? sgn * ratio * (COMP ? 1.f : kDebias) : 0.f;                  // cG = scale gamma
                     cf[2 * MAXD + 2] = __int_as_float(active ? d - 1 : -1);
                     cf[2 * MAXD + 3] = __int_as_float(active ? node * p.H * p.DV : 0);        // offset of the node's row
                 }
@@ -1215,9 +1354,44 @@ bool factorized_supported(const speca_dims *d)
 
 bool factorized_fused_supported(const speca_dims *d) { return factorized_supported(d) && d->max_depth <= kMaxDepth; }
 
-int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st)
+namespace {
+
+struct DeviceState { int sm_count; bool attr_set; };
+DeviceState g_device[64] = {};
+int g_withhold_first_load = 0;
+
+template <int TP, bool FUSED, int DK, bool DEEP, bool COMP>
+cudaError_t opt_in_smem()
+{
+    return cudaFuncSetAttribute(verify_factorized_kernel<TP, FUSED, DK, DEEP, COMP>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+template <bool FUSED, bool DEEP, bool COMP>
+void launch_one(bool one_tile, int d_k, int grid, cudaStream_t st, const CUtensorMap &map, const KQMaps &kq, const FParams &fp)
+{
+    constexpr int threads = FUSED ? kThreadsFused : (COMP ? kThreadsComp : kThreads);
+    if (d_k == kDK) {
+        if (one_tile) verify_factorized_kernel<1, FUSED, 128, DEEP, COMP><<<grid, threads, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, FUSED, 128, DEEP, COMP><<<grid, threads, kSmemBytes, st>>>(map, kq, fp);
+    } else {
+        if (one_tile) verify_factorized_kernel<1, FUSED, 256, DEEP, COMP><<<grid, threads, kSmemBytes, st>>>(map, kq, fp);
+        else verify_factorized_kernel<2, FUSED, 256, DEEP, COMP><<<grid, threads, kSmemBytes, st>>>(map, kq, fp);
+    }
+}
+
+}  // namespace
+
+// Test hook of the failure-detection test (not part of the public header): with `on` the producer of CTA 0
+// never requests its first state slice, so that CTA's bounded waits run out and the call reports
+// SPECA_STATUS_TIMEOUT.  Plain (non-fused) verification only.
+void factorized_set_withhold(int on) { g_withhold_first_load = on; }
+
+// comp: the compensated (fp32-grade) form; fused: commit-and-verify in one pass (single TF32 pass only).
+int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cudaStream_t st)
 {
     if (d_k != kDK && d_k != 2 * kDK) return int(cudaErrorInvalidValue);
+    if (fused && comp) return int(cudaErrorInvalidValue);
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return int(cudaErrorNotSupported);
     const long n_units = long(p.L) * p.B * p.H;
@@ -1256,70 +1430,49 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t 
         }
     }
 
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (sm_count <= 0) sm_count = 148;
+    // the SM count and the opt-in to large dynamic shared memory belong to a device, not to the process
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return int(cudaErrorInvalidDevice);
+    DeviceState &ds = g_device[dev];
+    if (ds.sm_count == 0) {
+        int n = 0;
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        ds.sm_count = n > 0 ? n : 148;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
-        const void *kernels[] = {
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 128>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 128>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 128>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 128>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, true, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, true, 256>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 128, true>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 128, true>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<1, false, 256, true>),
-            reinterpret_cast<const void *>(verify_factorized_kernel<2, false, 256, true>)};
-        for (const void *k : kernels) {
-            cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-            if (e != cudaSuccess) return int(e);
-        }
-        attr_set = true;
+    if (!ds.attr_set) {
+        cudaError_t e[] = {
+            opt_in_smem<1, false, 128, false, false>(), opt_in_smem<2, false, 128, false, false>(),
+            opt_in_smem<1, false, 256, false, false>(), opt_in_smem<2, false, 256, false, false>(),
+            opt_in_smem<1, true, 128, false, false>(),  opt_in_smem<2, true, 128, false, false>(),
+            opt_in_smem<1, true, 256, false, false>(),  opt_in_smem<2, true, 256, false, false>(),
+            opt_in_smem<1, false, 128, true, false>(),  opt_in_smem<2, false, 128, true, false>(),
+            opt_in_smem<1, false, 256, true, false>(),  opt_in_smem<2, false, 256, true, false>(),
+            opt_in_smem<1, false, 128, false, true>(),  opt_in_smem<2, false, 128, false, true>(),
+            opt_in_smem<1, false, 256, false, true>(),  opt_in_smem<2, false, 256, false, true>(),
+            opt_in_smem<1, false, 128, true, true>(),   opt_in_smem<2, false, 128, true, true>(),
+            opt_in_smem<1, false, 256, true, true>(),   opt_in_smem<2, false, 256, true, true>()};
+        for (cudaError_t x : e)
+            if (x != cudaSuccess) return int(x);
+        ds.attr_set = true;
     }
     FParams fp;
     fp.p = p;
     fp.n_units = n_units;
-    // Failure-detection test hook (plain verification only): with SPECA_TEST_WITHHOLD_FIRST_LOAD=1 in the environment one
-    // CTA's first state slice never arrives; its bounded waits expire, it reports SPECA_STATUS_TIMEOUT and exits cleanly.
-    const char *hook = getenv("SPECA_TEST_WITHHOLD_FIRST_LOAD");
-    fp.withhold_first_load = (hook != nullptr && hook[0] == '1') ? 1 : 0;
+    fp.withhold_first_load = g_withhold_first_load;
     // consecutive heads of one (layer, sequence) a CTA takes together: as many as divide H while
     // every SM still gets a group
     fp.heads_per_group = 1;
     for (int hg = 4; hg > 1; hg >>= 1)
-        if (p.H % hg == 0 && n_units / hg >= sm_count) { fp.heads_per_group = hg; break; }
+        if (p.H % hg == 0 && n_units / hg >= ds.sm_count) { fp.heads_per_group = hg; break; }
     const long n_groups = n_units / fp.heads_per_group;
-    const int grid = int(n_groups < sm_count ? n_groups : sm_count);
+    const int grid = int(n_groups < ds.sm_count ? n_groups : ds.sm_count);
     const bool one_tile = p.DV == kTileRows;
-    if (fused && d_k == kDK) {
-        if (one_tile) verify_factorized_kernel<1, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, true, 128><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
-    } else if (fused) {
-        if (one_tile) verify_factorized_kernel<1, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, true, 256><<<grid, kThreadsFused, kSmemBytes, st>>>(map, kq, fp);
-    } else if (p.max_depth > kMaxDepth) {
-        if (d_k == kDK) {
-            if (one_tile) verify_factorized_kernel<1, false, 128, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-            else verify_factorized_kernel<2, false, 128, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-        } else {
-            if (one_tile) verify_factorized_kernel<1, false, 256, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-            else verify_factorized_kernel<2, false, 256, true><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-        }
-    } else if (d_k == kDK) {
-        if (one_tile) verify_factorized_kernel<1, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, false, 128><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-    } else {
-        if (one_tile) verify_factorized_kernel<1, false, 256><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-        else verify_factorized_kernel<2, false, 256><<<grid, kThreads, kSmemBytes, st>>>(map, kq, fp);
-    }
+    const bool deep = p.max_depth > kMaxDepth;
+    if (fused) launch_one<true, false, false>(one_tile, d_k, grid, st, map, kq, fp);
+    else if (comp && deep) launch_one<false, true, true>(one_tile, d_k, grid, st, map, kq, fp);
+    else if (comp) launch_one<false, false, true>(one_tile, d_k, grid, st, map, kq, fp);
+    else if (deep) launch_one<false, true, false>(one_tile, d_k, grid, st, map, kq, fp);
+    else launch_one<false, false, false>(one_tile, d_k, grid, st, map, kq, fp);
     return int(cudaGetLastError());
 }
 

@@ -100,7 +100,8 @@ int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
 int launch_commit(const Params &p, int d_k, cudaStream_t st);
 bool factorized_supported(const speca_dims *d);
 bool factorized_fused_supported(const speca_dims *d);
-int launch_verify_factorized(const Params &p, int d_k, bool fused, cudaStream_t st);
+int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cudaStream_t st);
+void factorized_set_withhold(int on);
 bool effective_supported(const speca_dims *d);
 int launch_verify_effective(const Params &p, int d_k, cudaStream_t st);
 void effective_set_withhold(int on);

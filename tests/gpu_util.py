@@ -6,14 +6,28 @@ import torch
 from paper_2607_16673_b200 import binding as speca
 from paper_2607_16673_b200 import synth
 
-# Parity bar of the benchmark spec: outputs and committed states within 2e-3 of the
-# fp64 oracle, measured as max |x - r| / (|r| + rms(r)) over one output tensor (a
-# pure element-wise relative error is meaningless where outputs cross zero).
+# Parity bar of the method's acceptance criterion: outputs and committed states within 2e-3 of the fp64
+# oracle, measured as max |x - r| / (|r| + rms(r)) over one output tensor (a pure element-wise relative error
+# is meaningless where outputs cross zero).  Only the single-pass TF32 route (ROUTE_TF32) is held to this bar.
 TOL = 2e-3
-# fp32 kernels (state-resident serial route, decode, commit): every element is a
-# sum of <= d_k + depth products of O(1) terms accumulated in fp32; with d_k = 256
-# and depth 16 a loose bound is 300 * 2^-24 ~ 2e-5 relative to the tensor's scale.
+# Everything else computes with fp32 accuracy (the serial kernels, decode, commit, and the tensor-core routes
+# whose operands are split into a TF32 head and its exact remainder): every element is a sum of <= d_k + depth
+# products of O(1) terms accumulated in fp32; with d_k = 256 and depth 16 a loose bound is
+# 300 * 2^-24 ~ 2e-5 relative to the tensor's scale.
 TOL_FP32 = 2e-5
+
+
+def tol_for(route) -> float:
+    return TOL if route == speca.ROUTE_TF32 else TOL_FP32
+
+
+def max_err_over_max(x, r) -> float:
+    """Second figure reported beside rel_err: max |x - r| / max |r| over the tensor."""
+    x = np.asarray(x, dtype=np.float64)
+    r = np.asarray(r, dtype=np.float64)
+    if r.size == 0:
+        return 0.0
+    return float(np.max(np.abs(x - r)) / (np.max(np.abs(r)) + 1e-300))
 
 
 def rel_err(x, r) -> float:

@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2607_16673_b200 import binding as speca
 from paper_2607_16673_b200 import synth
-from gpu_util import DevProblem, TOL, TOL_FP32, rel_err
+from gpu_util import DevProblem, TOL, TOL_FP32, rel_err, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -77,13 +77,16 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("route", [speca.ROUTE_TF32, speca.ROUTE_AUTO], ids=["one-pass-tf32", "auto"])
 @pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
-def test_fused_equals_commit_then_verify(case):
+def test_fused_equals_commit_then_verify(case, route):
+    """ROUTE_TF32: the one-pass kernel (state read once as TF32).  AUTO: the commit kernel followed by the
+    fp32-grade verification, held to the fp32 bar."""
     name, L, H, d_v, mk_prev, mk_new = case
     rng = np.random.default_rng(11)
-    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(21, L, H, 128, d_v, mk_prev(rng), mk_new(rng), speca.ROUTE_FACTORIZED)
-    assert rel_err(cpu(S), S_ref) <= TOL, name
-    assert rel_err(cpu(d2.o), o_ref) <= TOL, name
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(21, L, H, 128, d_v, mk_prev(rng), mk_new(rng), route)
+    assert rel_err(cpu(S), S_ref) <= tol_for(route), name
+    assert rel_err(cpu(d2.o), o_ref) <= tol_for(route), name
     # sequences without an accepted path keep their state bit for bit
     for b in np.flatnonzero(p1.path_len == 0):
         assert torch.equal(S[:, b], d1.S[:, b])
@@ -93,8 +96,8 @@ def test_fused_equals_commit_then_verify(case):
     assert rel_err(cpu(S), cpu(d1.S)) <= 1e-4
 
 
-@pytest.mark.parametrize("route,with_u,tol", [(speca.ROUTE_SERIAL, True, TOL_FP32), (speca.ROUTE_FACTORIZED, False, TOL),
-                                              (speca.ROUTE_AUTO, True, TOL)])
+@pytest.mark.parametrize("route,with_u,tol", [(speca.ROUTE_SERIAL, True, TOL_FP32), (speca.ROUTE_TF32, False, TOL),
+                                              (speca.ROUTE_FACTORIZED, True, TOL_FP32), (speca.ROUTE_AUTO, True, TOL_FP32)])
 def test_fused_fallbacks_give_the_same_results(route, with_u, tol):
     """Serial route, or no u from the previous verification: the two kernels run back to back."""
     rng = np.random.default_rng(5)
@@ -120,7 +123,7 @@ def test_fused_key_width_256(d_v):
     rng = np.random.default_rng(13 + d_v)
     prev = synth.ragged_tree_batch(rng, 5, 4, 32, 8) + [synth.chain_parent(8), np.zeros(0, np.int32)]
     new = synth.ragged_tree_batch(rng, 5, 4, 32, 8) + [np.zeros(0, np.int32), synth.chain_parent(8)]
-    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(45, 2, 8, 256, d_v, prev, new, speca.ROUTE_AUTO, max_nodes=32)
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(45, 2, 8, 256, d_v, prev, new, speca.ROUTE_TF32, max_nodes=32)
     assert rel_err(cpu(d2.o), o_ref) <= TOL
     assert rel_err(cpu(S), S_ref) <= TOL
     d1.commit()
@@ -134,7 +137,7 @@ def test_nothing_pending_and_nothing_to_verify():
     prob = synth.make_problem(51, 2, 4, 128, 256, synth.ragged_tree_batch(rng, 3, 8, 30, 8))
     random_paths(rng, prob, zero_frac=0.0)
     # first round: no previous draft -> plain verification, S is not written
-    dp = DevProblem(prob, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    dp = DevProblem(prob, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     S = dp.S.clone()
     fused_call(dp, S, None, dp.path_idx, dp.path_len)
     assert dp.status_value() == 0 and torch.equal(S, dp.S)
@@ -142,7 +145,7 @@ def test_nothing_pending_and_nothing_to_verify():
     assert rel_err(cpu(dp.o), o_ref) <= TOL
     # last round: nothing left to verify -> plain commit of the pending paths
     empty = synth.make_problem(52, 2, 4, 128, 256, [np.zeros(0, np.int32)] * 3)
-    de = DevProblem(empty, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    de = DevProblem(empty, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     fused_call(de, S, prev_dict(dp), dp.path_idx, dp.path_len)
     assert de.status_value() == 0
     S_ref = oracle.commit(prob.S0, prob.k, prob.v, prob.alpha, prob.beta, prob.node_offsets, prob.path_idx, prob.path_len)
@@ -157,9 +160,9 @@ def test_bad_pending_path_skips_only_that_commit():
     p1 = synth.make_problem(61, 1, 4, 128, 256, parents)
     p2 = synth.make_problem(62, 1, 4, 128, 256, [synth.chain_parent(5)] * 3)
     synth._set_paths(p1, [[0, 1, 2], [0, 2, 3], synth.root_path(parents[2], 19)])      # sequence 1: 2 is not a child of 0
-    d1 = DevProblem(p1, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d1 = DevProblem(p1, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     d1.verify_tree()
-    d2 = DevProblem(p2, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d2 = DevProblem(p2, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     S = d1.S.clone()
     fused_call(d2, S, prev_dict(d1), d1.path_idx, d1.path_len)
     assert d2.status_value() == speca.STATUS_BAD_PATH
@@ -187,9 +190,9 @@ def test_rejected_new_tree_still_gets_its_commit():
     p2 = synth.make_problem(72, 1, 4, 128, 128, [synth.chain_parent(4)] * 2)
     synth._set_paths(p1, [[0, 1], [0, 1, 2]])
     p2.parent[5] = 3                      # sequence 1, local node 1: parent 3 >= 1 is not topological
-    d1 = DevProblem(p1, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d1 = DevProblem(p1, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     d1.verify_tree()
-    d2 = DevProblem(p2, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d2 = DevProblem(p2, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     S = d1.S.clone()
     speca.commit_verify_tree(d2.dims, S, prev_dict(d1), d1.path_idx, d1.path_len, d2.q, d2.k, d2.v, d2.alpha, d2.beta,
                              d2.node_offsets, d2.T, d2.parent, None, d2.o, d2.u, d2.ws, d2.status)
@@ -210,7 +213,7 @@ def test_fused_rounds_carry_the_state():
     for r in range(6):
         parents = synth.mixed_chain_tree_batch(rng, B, 8, 48, 8) if r % 2 == 0 else synth.ragged_tree_batch(rng, B, 4, 64, 8)
         probs.append(synth.make_problem(100 + r, L, H, 128, 256, parents))
-    devs = [DevProblem(p, route=speca.ROUTE_AUTO, want_u=True, max_nodes=64) for p in probs]
+    devs = [DevProblem(p, route=speca.ROUTE_TF32, want_u=True, max_nodes=64) for p in probs]
     S = devs[0].S.clone()
     S_ref = probs[0].S0.astype(np.float64)
     prev = None
@@ -246,7 +249,7 @@ def test_more_sequences_than_the_walk_table_holds():
     prev = [synth.random_tree_parent(int(rng.integers(1, 13)), 4, 3, rng) for _ in range(B)]
     new = [synth.random_tree_parent(int(rng.integers(1, 13)), 4, 3, rng) for _ in range(B)]
     new[140] = np.zeros(0, np.int32)
-    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(47, 1, 2, 128, 128, prev, new, speca.ROUTE_FACTORIZED, max_nodes=16)
+    p1, p2, d1, d2, S, S_ref, o_ref = run_pair(47, 1, 2, 128, 128, prev, new, speca.ROUTE_TF32, max_nodes=16)
     o1_ref = oracle.verify_tree(p1.S0, p1.q, p1.k, p1.v, p1.alpha, p1.beta, p1.node_offsets, p1.parent)
     assert rel_err(cpu(d1.o), o1_ref) <= TOL
     assert rel_err(cpu(d2.o), o_ref) <= TOL
@@ -267,11 +270,11 @@ def test_tensor_core_kernels_write_nothing_outside_their_tensors():
     p1 = synth.make_problem(191, 2, 3, 128, 256, synth.ragged_tree_batch(rng, 3, 5, 40, 8))
     p2 = synth.make_problem(192, 2, 3, 128, 256, synth.ragged_tree_batch(rng, 3, 5, 40, 8))
     random_paths(rng, p1, zero_frac=0.0)
-    d1 = DevProblem(p1, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d1 = DevProblem(p1, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     bo, d1.o = _banded(d1.o)
     bu, d1.u = _banded(d1.u)
     d1.verify_tree()
-    d2 = DevProblem(p2, route=speca.ROUTE_FACTORIZED, want_u=True, max_nodes=64)
+    d2 = DevProblem(p2, route=speca.ROUTE_TF32, want_u=True, max_nodes=64)
     bo2, d2.o = _banded(d2.o)
     bu2, d2.u = _banded(d2.u)
     bS, S = _banded(d1.S)
