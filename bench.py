@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the speculative verify -> accept -> commit path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4|paper256|trees64|chains8|paper] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4|cfg3|cfg2|paper256|trees64|chains8|paper]
+                    [--sweep commit-len|unit-types] [--impl reference]
 
 One "step" is one round of the whole hot path over one batch of synthetic draft input:
 plan + verify (all layers, heads, nodes) -> greedy accept -> commit, with the committed
@@ -52,11 +53,15 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS) + ["paper"],
+    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS) + ["paper", "cfg2", "cfg3"],
                     help="cfg5 (default), cfg4, paper256, trees64 / chains8 (cfg5's unit types on their own), or 'paper': "
                          "the paper's own target shape and proposal shapes (Table 1)")
     ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
-    ap.add_argument("--route", type=int, default=0, help="0 auto, 1 serial, 2 factorized")
+    ap.add_argument("--route", type=int, default=0,
+                    help="0 auto (fp32-grade), 1 serial, 2 factorised (fp32-grade), 3 single-pass TF32, 4 effective-query")
+    ap.add_argument("--sweep", default=None, choices=["commit-len", "unit-types"],
+                    help="commit-len: commit throughput against the accepted path length; unit-types: time per "
+                         "(layer, sequence, head) unit and SM of 8-token chains and 64-node trees, per route")
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -335,10 +340,25 @@ def run_speca(args):
     dec_bytes = L * B * H * (2 * 4 * dk * dv + 4 * dk + 2 * dv + 8 + 4 * dv)
     del S_dec
 
+    # --- the same verification on the single-pass TF32 route (context: opt-in, 2e-3-grade) ---------
+    dims_tf32 = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64 if dk <= 128 else 32, speca.ROUTE_TF32)
+    p0 = pool[0]
+    for _ in range(2):
+        speca.verify_tree(dims_tf32, S, p0["q"], p0["k"], p0["v"], p0["alpha"], p0["beta"], p0["d_offs"], p0["T"],
+                          p0["d_parent"], p0["d_depth"], o_view(p0["T"]), None, ws, status)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(5):
+        speca.verify_tree(dims_tf32, S, p0["q"], p0["k"], p0["v"], p0["alpha"], p0["beta"], p0["d_offs"], p0["T"],
+                          p0["d_parent"], p0["d_depth"], o_view(p0["T"]), None, ws, status)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    tf32_ms = e0.elapsed_time(e1) / 5
+
     # --- convolution-state commit (the other half of the state holder), same accepted paths --------
     ch, W = H * (2 * dk + dv), 3
     C = torch.zeros(L, B, W, ch, dtype=torch.bfloat16, device=dev)
-    p0 = pool[0]
     x_conv = torch.zeros(L, p0["T"], ch, dtype=torch.bfloat16, device=dev)
     speca.greedy_accept(B, 8, p0["d_offs"], p0["d_parent"], p0["d_draft"], p0["d_target"], p0["d_root"],
                         path_idx, path_len, next_tok, status)
@@ -429,11 +449,14 @@ def run_speca(args):
                    "d_k": dk, "d_v": dv, "nodes_per_step_per_gpu": [p["T"] for p in pool],
                    "mean_accepted_len": float(np.mean([p["path_len"].mean() for p in pool])),
                    "input_pool": POOL, "l2": f"inputs larger than L2 (state {L * B * H * dk * dv * 4 / 1e9:.1f} GB)",
-                   "route": args.route, "parallelism": f"dp{world} (sequences partitioned, no collective)"},
+                   "route": {0: "auto: tensor-core route with split operands (fp32-grade)", 1: "serial", 2: "factorised, split operands",
+                             3: "single-pass TF32", 4: "effective-query"}.get(args.route, str(args.route)),
+                   "parallelism": f"dp{world} (sequences partitioned, no collective)"},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC.get(dom) if args.workload == "cfg5" and not args.layers and not args.batch else None,
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic(args.workload, dom) if not args.layers and not args.batch else None,
                      "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms},
         "kernels": {"verify_ms": t_verify, "accept_ms": t_accept, "commit_ms": t_commit,
+                    "verify_single_pass_tf32_ms": tf32_ms,
                     "verify_gbs": vb / K / (t_verify * 1e-3) / 1e9, "commit_gbs": cb / K / (t_commit * 1e-3) / 1e9,
                     "step_gbs": (vb + cb) / K / (ms_per_step * 1e-3) / 1e9,
                     "step_frac_of_peak": (vb + cb) / K / (ms_per_step * 1e-3) / 1e9 / peak,
@@ -463,6 +486,9 @@ def run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, di
     round), then runs greedy acceptance.  Reported beside the headline, not instead of it."""
     import torch
     L, B, H, dk, dv = dims.n_layers, dims.batch, dims.heads, dims.d_k, dims.d_v
+    # the one-pass kernel exists on the single-pass TF32 route only (on the default route the entry point runs
+    # the commit kernel and then the fp32-grade verification, i.e. the separate step)
+    dims = speca.Dims(L, B, H, dk, dv, 1.0, dims.max_depth, dims.max_nodes, speca.ROUTE_TF32)
     Tmax = max(p["T"] for p in pool)
     u_buf = [torch.empty(L * Tmax * H * dv, dtype=torch.float32, device=dev) for _ in range(2)]
     paths = [(torch.zeros(B, 8, dtype=torch.int32, device=dev), torch.zeros(B, dtype=torch.int32, device=dev))
@@ -497,14 +523,15 @@ def run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, di
     ms = e0.elapsed_time(e1)
     assert int(status.item()) == 0, f"device status word {int(status.item())}"
     tokens = sum(pool[i % POOL]["T"] for i in range(W, W + K))
-    # algorithmic bytes: state read once, written once where something is committed, records in, o out,
-    # records of the accepted nodes; the u rows written and re-read are not counted
+    # bytes: state read once, written once where something is committed, records in, o out, keys and gates of the
+    # accepted nodes -- and the u rows, which every round writes for all nodes and re-reads for the accepted ones
     Sb = 4 * dk * dv
     nbytes = 0
     for i in range(W, W + K):
         p, pp = pool[i % POOL], pool[(i - 1) % POOL]
         nbytes += L * B * H * Sb + int(np.count_nonzero(pp["path_len"])) * L * H * Sb
         nbytes += p["T"] * L * H * (4 * dk + 2 * dv + 8 + 4 * dv) + int(pp["path_len"].sum()) * L * H * (2 * dk + 2 * dv + 8)
+        nbytes += p["T"] * L * H * 4 * dv + int(pp["path_len"].sum()) * L * H * 4 * dv
     if dist is not None:
         tt = torch.tensor([ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -515,13 +542,26 @@ def run_fused(args, speca, dims, S, pool, o_buf, ws, status, stream, barrier, di
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"value": tokens * L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / K, "steps": K, "gpu_launches": 4 * K,
             "algorithmic_gbs": gbs, "frac_of_peak": gbs / peak, "peak_kind": f"of {peak_kind}",
+            "route": "single-pass TF32 (SPECA_ROUTE_TF32): outputs within the 2e-3 bar, not fp32-grade",
             "note": "speca_commit_verify_tree + speca_greedy_accept per round; the commit of round r runs inside the "
-                    "verification of round r+1 (state read once and written once per round)"}
+                    "verification of round r+1 (state read once and written once per round); the u rows written and "
+                    "re-read are counted in algorithmic_gbs"}
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant
-# kernels from the ncu captures summarised under profiles/; None until captured.
-NCU_TRAFFIC = {"verify": 12 * 835.1e6, "commit": 12 * 716.9e6}     # 2-layer captures x 12 (traffic is proportional to units)
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel, from the ncu
+    captures summarised in profiles/dram_traffic.md: rows `| workload | kernel | captured bytes | scale | ... |`,
+    the capture being a reduced-layer case scaled to the full launch by the number of units.  None if absent."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
+    try:
+        with open(path) as f:
+            for line in f:
+                cells = [c.strip() for c in line.strip().strip("|").split("|")]
+                if len(cells) >= 4 and cells[0] == workload and cells[1] == kernel:
+                    return float(cells[2]) * float(cells[3])
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def run_e2e(args, speca, dims, S, pool, o_buf, ws, status, path_idx, path_len, next_tok, stream):
@@ -628,7 +668,21 @@ def cpu_baseline(workload: str, L: int, H: int, dk: int, dv: int, n_units: int =
     dt = sum(time_oracle_once(prob) for _ in range(passes))
     # one unit is 1/H of a token-layer
     value = passes * prob.T / H / dt
-    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    # the same oracle on one thread, on a sixteenth of the sample
+    small = oracle_sample_problem(workload, H, dk, dv, max(8, n_units // 16), seed=4343)
+    cores = oracle.num_threads()
+    prev_env = os.environ.get("OMP_NUM_THREADS")
+    single = None
+    try:
+        oracle.set_num_threads(1)
+        t1 = time_oracle_once(small)
+        single = small.T / H / t1
+    except AttributeError:
+        pass
+    finally:
+        if hasattr(oracle, "set_num_threads"):
+            oracle.set_num_threads(cores)
+    return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "single_thread_value": single,
             "sample": f"{passes} passes over {n_units} (layer, sequence, head) units of {workload} ({prob.T} node-units "
                       f"per pass), verify+accept+commit, {dt:.1f} s of CPU work, scaled by 1/heads to token-layers"}
 
@@ -777,12 +831,221 @@ def run_paper_shapes(args):
                 "is context only: r2l_replay_ms here replays the recurrent layer alone through speca_verify_chain"}))
 
 
+
+# ---------------------------------------------------------------------------
+# the two small single-sequence configurations (latency-bound: 384 units on 148 SMs, 24 MiB of state)
+# ---------------------------------------------------------------------------
+def run_small(args):
+    """cfg2: 1 sequence x 24 layers x 16 heads, d_k = d_v = 128, a chain of 8 draft tokens, accepted length drawn
+    uniformly from 0..8 per step, beside the same 8 tokens by 8 speca_decode_step calls.  cfg3: the same shape with a
+    32-node tree (depth <= 6) and a random root-to-leaf accepted path.  The 24 MiB state fits L2, so eight copies
+    are rotated (192 MiB, larger than L2) and the L2-resident figure (one copy) is reported beside it.  Also
+    reported: what one call costs the host (enqueue time with the GPU kept busy)."""
+    import torch
+    from paper_2607_16673_b200 import binding as speca
+    from paper_2607_16673_b200 import synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    L, H, dk, dv, COPIES = args.layers or 24, 16, 128, 128, 8
+    chain = args.workload == "cfg2"
+    rng = np.random.default_rng(2 if chain else 3)
+    par = synth.chain_parent(8) if chain else synth.random_tree_parent(32, 6, 4, rng)
+    n = len(par)
+    prob = synth.make_problem(20 + n, L, H, dk, dv, [par], max_depth=8)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    bf = lambda a: t(a.view(np.int16)).view(torch.bfloat16)
+    dims = speca.Dims(L, 1, H, dk, dv, 1.0, 8, 8 if chain else 32, args.route)
+    S = [t(prob.S0) + 0 for _ in range(COPIES)]
+    q, k, v, al, be = bf(prob.q), bf(prob.k), bf(prob.v), t(prob.alpha), t(prob.beta)
+    offs, parent = t(prob.node_offsets), t(prob.parent)
+    draft, target, root = t(prob.draft_tok), t(prob.target_tok), t(prob.root_target_tok)
+    o = torch.empty(L, n, H, dv, device=dev)
+    ws = speca.alloc_workspace(dims, n, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    # accepted paths: cfg2 a prefix of length 0..8 per step, cfg3 a random root-to-leaf path
+    NP = 16
+    has_child = np.zeros(n, dtype=bool)
+    has_child[par[par >= 0]] = True
+    leaves = np.flatnonzero(~has_child)
+    paths_h = [list(range(int(rng.integers(0, 9)))) if chain else synth.root_path(par, int(rng.choice(leaves)))
+               for _ in range(NP)]
+    pidx = [torch.full((1, 8), -1, dtype=torch.int32, device=dev) for _ in range(NP)]
+    plen = [torch.tensor([len(p_)], dtype=torch.int32, device=dev) for p_ in paths_h]
+    for j, p_ in enumerate(paths_h):
+        if p_:
+            pidx[j][0, :len(p_)] = t(np.asarray(p_, np.int32))
+    gp = torch.full((1, 8), -1, dtype=torch.int32, device=dev)
+    gl = torch.zeros(1, dtype=torch.int32, device=dev)
+    gn = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def verify(Sx):
+        if chain:
+            speca.verify_chain(dims, Sx, q, k, v, al, be, offs, n, o, None, ws, status)
+        else:
+            speca.verify_tree(dims, Sx, q, k, v, al, be, offs, n, parent, None, o, None, ws, status)
+
+    def step(i, copies):
+        Sx = S[i % copies]
+        verify(Sx)
+        speca.greedy_accept(1, 8, offs, parent, draft, target, root, gp, gl, gn, status)
+        speca.commit(dims, Sx, k, v, al, be, offs, n, parent, pidx[i % NP], plen[i % NP], status)
+
+    def timed(fn, reps):
+        for i in range(max(3, args.warmup)):
+            fn(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        w0 = time.perf_counter()
+        e0.record(stream)
+        for i in range(reps):
+            fn(i)
+        e1.record(stream)
+        w1 = time.perf_counter()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps, (w1 - w0) / reps * 1e6
+
+    K = max(args.steps, 20)
+    sampler = ClockSampler(0)
+    sampler.mark()
+    ms_step, _ = timed(lambda i: step(i, COPIES), K)
+    sampler.mark()
+    clocks = sampler.stop()
+    ms_step_l2, _ = timed(lambda i: step(i, 1), K)
+    ms_verify, us_verify_host = timed(lambda i: verify(S[i % COPIES]), K)
+    ms_verify_l2, _ = timed(lambda i: verify(S[0]), K)
+    ms_commit, us_commit_host = timed(lambda i: speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent,
+                                                            pidx[i % NP], plen[i % NP], status), K)
+    # the same tokens one at a time: n decode steps (chain order; for the tree, its first root-to-leaf path)
+    d1 = speca.Dims(L, 1, H, dk, dv)
+    order = list(range(n)) if chain else paths_h[0]
+    qs = [q[:, j:j + 1].contiguous() for j in order]
+    ks = [k[:, j:j + 1].contiguous() for j in order]
+    vs = [v[:, j:j + 1].contiguous() for j in order]
+    als = [al[:, j:j + 1].contiguous() for j in order]
+    bes = [be[:, j:j + 1].contiguous() for j in order]
+    o1 = torch.empty(L, 1, H, dv, device=dev)
+
+    def decode_all(i):
+        Sx = S[i % COPIES]
+        for j in range(len(order)):
+            speca.decode_step(d1, Sx, qs[j], ks[j], vs[j], als[j], bes[j], o1)
+
+    ms_decode, _ = timed(decode_all, K)
+    assert int(status.item()) == 0
+    mean_acc = float(np.mean([len(p_) for p_ in paths_h]))
+    Sb = 4 * dk * dv
+    units = L * H
+    vbytes = units * Sb + n * units * (4 * dk + 2 * dv + 8 + 4 * dv)
+    cbytes = 2 * units * Sb * float(np.mean([len(p_) > 0 for p_ in paths_h])) + mean_acc * units * (2 * dk + 2 * dv + 8)
+    peak, peak_kind = measured_peak_gbs()
+    achieved = (vbytes + cbytes) / (ms_step * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": n * L / (ms_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: 1 seq x {L} layers x {H} heads, d_k=d_v=128; " +
+                               ("chain of 8, accepted length uniform 0..8" if chain else
+                                f"{n}-node tree (depth {int(synth.depth_of(par).max())}), random root-to-leaf path"),
+                   "l2": f"{COPIES} rotating copies of the {units * Sb / 2**20:.0f} MiB state (larger than L2)",
+                   "route": args.route, "mean_accepted_len": mean_acc},
+        "roofline": {"bound": "hbm", "kernel": "step", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "note": "latency-bound: 384 units on 148 SMs, a few tens of MB per call"},
+        "latency_ms": {"step": ms_step, "step_l2_resident": ms_step_l2, "plan_verify": ms_verify,
+                       "plan_verify_l2_resident": ms_verify_l2, "commit": ms_commit,
+                       "same_tokens_by_decode_steps": ms_decode, "decode_steps": len(order)},
+        "host_us_per_call": {"verify": us_verify_host, "commit": us_commit_host,
+                             "note": "wall time to enqueue one call (Python binding + C entry point) with the GPU busy"},
+        "gpu_launches": (3 if chain and args.route == 1 else 4) * K,
+        "clocks": clocks,
+    }
+    print(json.dumps(out))
+
+
+# ---------------------------------------------------------------------------
+# sweeps behind the figures in DESIGN.md
+# ---------------------------------------------------------------------------
+def run_sweep(args):
+    import torch
+    from paper_2607_16673_b200 import binding as speca
+    from paper_2607_16673_b200 import synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    L, B, H, dk, dv = args.layers or 24, args.batch or 128, 16, 128, 256
+    peak, peak_kind = measured_peak_gbs()
+    t = lambda a: torch.from_numpy(a).to(dev)
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    S = synth.device_state(1, L, B, H, dk, dv, 0.02, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rows = []
+    if args.sweep == "commit-len":
+        # every sequence an 8-token chain, the first A tokens accepted
+        hi = host_round_inputs("chains8", B, 5000)
+        q, k, v, al, be = synth.device_records(7, L, hi["T"], H, dk, dv, dev)
+        dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, args.route)
+        offs, par = t(hi["node_offsets"]), t(hi["parent"])
+        for A in (1, 2, 4, 8):
+            pidx = torch.arange(8, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()
+            plen = torch.full((B,), A, dtype=torch.int32, device=dev)
+            ms = timed(lambda: speca.commit(dims, S, k, v, al, be, offs, hi["T"], par, pidx, plen, status))
+            nbytes = 2 * L * B * H * 4 * dk * dv + A * B * L * H * (2 * dk + 2 * dv + 8)
+            rows.append({"accepted": A, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peak})
+    else:
+        sm = torch.cuda.get_device_properties(dev).multi_processor_count
+        for wl in ("chains8", "trees64"):
+            hi = host_round_inputs(wl, B, 5000)
+            q, k, v, al, be = synth.device_records(7, L, hi["T"], H, dk, dv, dev)
+            offs, par = t(hi["node_offsets"]), t(hi["parent"])
+            o = torch.empty(L, hi["T"], H, dv, device=dev)
+            for name, route in (("default (fp32-grade)", 0), ("single-pass TF32", 3), ("effective-query", 4)):
+                dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, route)
+                ws = speca.alloc_workspace(dims, hi["T"], dev)
+                ms = timed(lambda: speca.verify_tree(dims, S, q, k, v, al, be, offs, hi["T"], par, None, o, None, ws, status))
+                nbytes = L * B * H * 4 * dk * dv + hi["T"] * L * H * (4 * dk + 2 * dv + 8 + 4 * dv)
+                rows.append({"units": wl, "route": name, "verify_ms": ms, "us_per_unit_per_sm": ms * 1e3 / (L * B * H / sm),
+                             "gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peak})
+    assert int(status.item()) == 0
+    print(json.dumps({"sweep": args.sweep, "shape": f"{B} seq x {L} layers x {H} heads, d_k={dk} d_v={dv}",
+                      "peak_gbs": peak, "peak_kind": peak_kind, "rows": rows}))
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script, one process per GPU."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args))
+    if args.sweep and args.impl != "reference":
+        run_sweep(args)
+        return
+    if args.workload in ("cfg2", "cfg3") and args.impl != "reference":
+        run_small(args)
+        return
     if args.workload == "paper" and args.impl != "reference":
         run_paper_shapes(args)
         return
-    if args.impl == "reference" and args.workload == "paper":
+    if args.impl == "reference" and args.workload in ("paper", "cfg2", "cfg3"):
         args.workload = "cfg5"
     if args.impl == "reference":
         run_reference(args)

@@ -94,6 +94,11 @@ def num_threads() -> int:
     return int(_load().oracle_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """Threads the loops over independent units may use (for timing; results do not depend on it)."""
+    _load().oracle_set_num_threads(int(n))
+
+
 def decode_step(S, q, k, v, alpha, beta, scale: float = 1.0):
     """One token per sequence.  S [L,B,H,dv,dk]; q,k uint16 [L,B,H,dk]; v uint16 [L,B,H,dv].
 

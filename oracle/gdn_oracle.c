@@ -100,6 +100,16 @@ int oracle_num_threads(void)
 #endif
 }
 
+/* Threads the unit loops below may use (timing only: no result depends on it). */
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* Single-token decode step for every (layer, sequence, head): T == B, one token
  * per sequence.  S is updated in place, o = scale * S_new q. */
 int oracle_decode_step(int L, int B, int H, int d_k, int d_v, double scale,

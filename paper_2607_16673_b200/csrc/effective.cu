@@ -846,18 +846,22 @@ verify_effective_kernel(const __grid_constant__ CUtensorMap s0_map, const __grid
                 const int s = it % NS;
                 const uint32_t ph = (it / NS) & 1;
                 if (!(ok = WAIT(0, bar(kFull + s), ph))) break;
-                if (!(ok = WAIT(1, bar(kP1Done + s), ph))) break;
                 if (e >= TP && e < 2 * TP) {                     // value tiles are not split
+                    if (!(ok = WAIT(1, bar(kP1Done + s), ph))) break;
                     warp_arrive(bar(kLo + s), lane);
                     continue;
                 }
+                // the remainders are formed while the first products are still reading the slice; only the stores wait
                 float4 *sl = reinterpret_cast<float4 *>(smem + LY::OffRing + s * kSliceBytes);
+                float4 v[kSliceBytes / 16 / 128];
 #pragma unroll
                 for (int k = 0; k < kSliceBytes / 16 / 128; ++k) {
-                    float4 v = sl[stid + k * 128];
-                    v.x = tf32_rest(v.x); v.y = tf32_rest(v.y); v.z = tf32_rest(v.z); v.w = tf32_rest(v.w);
-                    sl[stid + k * 128] = v;
+                    v[k] = sl[stid + k * 128];
+                    v[k].x = tf32_rest(v[k].x); v[k].y = tf32_rest(v[k].y); v[k].z = tf32_rest(v[k].z); v[k].w = tf32_rest(v[k].w);
                 }
+                if (!(ok = WAIT(1, bar(kP1Done + s), ph))) break;
+#pragma unroll
+                for (int k = 0; k < kSliceBytes / 16 / 128; ++k) sl[stid + k * 128] = v[k];
                 fence_proxy_async();
                 warp_arrive(bar(kLo + s), lane);
             }

@@ -649,6 +649,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         Unit x;
         bool ok = mt < TP;
         const uint32_t bop = sbase + kOffBop, stage = sbase + kOffStage;
+        PROF_DECL
         auto issue_gram = [&](uint32_t seq, int npad) -> bool {
             const int pr = seq & 1;
             if (!wait_fast(bar(kBarStageReady), seq & 1, abort_flag)) return false;
@@ -673,10 +674,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         while (have && ok) {
             const int pr = unit_seq & 1;
             const uint32_t acc = tmem_base + pr * kPairCols + mt * kAccCols;
-            if (!(ok = wait_fast(bar(kBarBReady), unit_seq & 1, abort_flag))) break;
+            if (!(ok = WAIT(0, bar(kBarBReady), unit_seq & 1))) break;
             if (mt == 0) {
-                if (!(ok = wait_fast(bar(kBarGramDone), unit_seq & 1, abort_flag))) break;
-            } else if (!(ok = wait_fast(bar(kBarPairFree + pr), ((unit_seq >> 1) & 1) ^ 1, abort_flag))) {
+                if (!(ok = WAIT(1, bar(kBarGramDone), unit_seq & 1))) break;
+            } else if (!(ok = WAIT(1, bar(kBarPairFree + pr), ((unit_seq >> 1) & 1) ^ 1))) {
                 break;
             }
             tc_fence_after();
@@ -688,7 +689,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     const uint32_t it = (unit_seq * NC + c) * TP + mt;
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1;
-                    if (!(ok = wait_fast(bar(kBarFull + s), ph, abort_flag))) break;
+                    if (!(ok = WAIT(2, bar(kBarFull + s), ph))) break;
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t sa = sbase + kOffRing + s * kStageBytes;
@@ -699,7 +700,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     }
                     __syncwarp();
                     if (ps >= 0) {
-                        if (!(ok = wait_fast(bar(kBarLo + ps), pph, abort_flag))) break;
+                        if (!(ok = WAIT(3, bar(kBarLo + ps), pph))) break;
                         tc_fence_after();
                         if (lane == 0) {
                             const uint32_t sa = sbase + kOffRing + ps * kStageBytes;
@@ -713,7 +714,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     ps = s; pph = ph;
                 } else {
                     // the last slice's second pass closes the tile
-                    if (!(ok = wait_fast(bar(kBarLo + ps), pph, abort_flag))) break;
+                    if (!(ok = WAIT(3, bar(kBarLo + ps), pph))) break;
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t sa = sbase + kOffRing + ps * kStageBytes;
@@ -732,6 +733,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             have = next_unit(walk, x);
             if (have && mt == 0) ok = issue_gram(unit_seq, x.npad);
         }
+        PROF_STORE()
         // everything this warp issued must have completed before TMEM is released
         if (mt < TP) {
             if (lane == 0) mma_commit(bar(kBarDrain));
@@ -744,27 +746,32 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
         uint32_t it = 0;
         Unit x;
         bool ok = true;
+        PROF_DECL
         for (bool have = first_unit(walk, x); have && ok; have = next_unit(walk, x)) {
             for (int i = 0; i < TP * NC; ++i, ++it) {
                 const int s = it % NS;
                 const uint32_t ph = (it / NS) & 1;
-                if (!(ok = wait_fast(bar(kBarFull + s), ph, abort_flag))) break;
-                if (!(ok = wait_fast(bar(kBarP1Done + s), ph, abort_flag))) break;
+                // the remainders are formed while the first pass is still reading the slice; only the stores wait
+                if (!(ok = WAIT(0, bar(kBarFull + s), ph))) break;
                 float4 *sl = reinterpret_cast<float4 *>(smem + kOffRing + s * kStageBytes);
+                float4 v[kStageBytes / 16 / 128];
 #pragma unroll
                 for (int k = 0; k < kStageBytes / 16 / 128; ++k) {
-                    float4 v = sl[stid + k * 128];
-                    v.x -= __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
-                    v.y -= __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
-                    v.z -= __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
-                    v.w -= __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
-                    sl[stid + k * 128] = v;
+                    v[k] = sl[stid + k * 128];
+                    v[k].x -= __uint_as_float(__float_as_uint(v[k].x) & 0xffffe000u);
+                    v[k].y -= __uint_as_float(__float_as_uint(v[k].y) & 0xffffe000u);
+                    v[k].z -= __uint_as_float(__float_as_uint(v[k].z) & 0xffffe000u);
+                    v[k].w -= __uint_as_float(__float_as_uint(v[k].w) & 0xffffe000u);
                 }
+                if (!(ok = WAIT(1, bar(kBarP1Done + s), ph))) break;
+#pragma unroll
+                for (int k = 0; k < kStageBytes / 16 / 128; ++k) sl[stid + k * 128] = v[k];
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarLo + s));
             }
         }
+        PROF_STORE()
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
         uint32_t it = 0, unit_seq = 0;
