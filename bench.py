@@ -912,10 +912,25 @@ def run_small(args):
     sampler.mark()
     clocks = sampler.stop()
     ms_step_l2, _ = timed(lambda i: step(i, 1), K)
-    ms_verify, us_verify_host = timed(lambda i: verify(S[i % COPIES]), K)
+    def host_us(fn, reps=50):
+        """Wall time the host spends inside one call, the GPU idle beforehand (so the launch queue never blocks)."""
+        tot = 0.0
+        for i in range(reps + 5):
+            torch.cuda.synchronize()
+            w0 = time.perf_counter()
+            fn(i)
+            w1 = time.perf_counter()
+            if i >= 5:
+                tot += w1 - w0
+        torch.cuda.synchronize()
+        return tot / reps * 1e6
+
+    ms_verify, _ = timed(lambda i: verify(S[i % COPIES]), K)
+    us_verify_host = host_us(lambda i: verify(S[i % COPIES]))
     ms_verify_l2, _ = timed(lambda i: verify(S[0]), K)
-    ms_commit, us_commit_host = timed(lambda i: speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent,
-                                                            pidx[i % NP], plen[i % NP], status), K)
+    commit_fn = lambda i: speca.commit(dims, S[i % COPIES], k, v, al, be, offs, n, parent, pidx[i % NP], plen[i % NP], status)
+    ms_commit, _ = timed(commit_fn, K)
+    us_commit_host = host_us(commit_fn)
     # the same tokens one at a time: n decode steps (chain order; for the tree, its first root-to-leaf path)
     d1 = speca.Dims(L, 1, H, dk, dv)
     order = list(range(n)) if chain else paths_h[0]
@@ -956,7 +971,8 @@ def run_small(args):
                        "plan_verify_l2_resident": ms_verify_l2, "commit": ms_commit,
                        "same_tokens_by_decode_steps": ms_decode, "decode_steps": len(order)},
         "host_us_per_call": {"verify": us_verify_host, "commit": us_commit_host,
-                             "note": "wall time to enqueue one call (Python binding + C entry point) with the GPU busy"},
+                             "note": "wall time of one call on the host (Python binding + C entry point: argument checks, tensor maps, "
+                                     "launches), GPU idle beforehand"},
         "gpu_launches": (3 if chain and args.route == 1 else 4) * K,
         "clocks": clocks,
     }

@@ -47,7 +47,8 @@
  * device memory (bad parent pointer, offsets that decrease, a sequence larger
  * than dims.max_nodes or deeper than dims.max_depth, an accepted path that is
  * not a parent chain, a bounded wait that expired) make the kernels skip the
- * affected sequence -- its outputs and its state stay untouched -- and OR a
+ * affected sequence -- its outputs and its state stay untouched (one exception: an expired wait inside the
+ * one-pass speca_commit_verify_tree, see there) -- and OR a
  * SPECA_STATUS_* bit into *status_word, a device int32 the caller zeroes
  * beforehand and reads back when it wants to know.  No kernel traps.
  */
@@ -119,7 +120,8 @@ int         speca_version(void);
 const char *speca_strerror(int code);
 
 /* Bytes of caller-provided device scratch the verify calls need for `total_nodes`
- * packed nodes (topology plan shared by all layers and heads).  Never 0. */
+ * packed nodes (topology plan shared by all layers and heads).  Positive for valid arguments; 0 if dims is NULL,
+ * dims->batch < 1 or total_nodes < 0. */
 size_t speca_workspace_bytes(const speca_dims *dims, int32_t total_nodes);
 
 /* Single-token decode step, the autoregressive baseline (Section 2.2: every step
@@ -224,12 +226,15 @@ int speca_commit(const speca_dims *dims, float *S,
  * u_or_null to be able to fuse the next round; it must not be the buffer u_prev_or_null
  * points to, and o / u must not alias any input.
  *
- * The single-pass kernel runs when the tensor-core route applies with max_depth <= 8
- * (d_v in {128, 256}; d_k = 128 with max_nodes <= 64 or d_k = 256 with max_nodes <= 32;
- * route != SERIAL) and u_prev_or_null is given: the pending update is then S <- gamma_A S + sum_i (gamma_A / gamma_i) u_i k_i^T,
- * which needs only u, k and alpha of the accepted nodes (v_prev and beta_prev are not
- * read).  Otherwise the commit and verify kernels are launched back to back on `stream`
- * with the same results.  workspace_bytes must be at least speca_workspace_bytes(). */
+ * One pass or two.  With dims.route = SPECA_ROUTE_TF32, a shape that route takes with max_depth <= 8 (d_v in
+ * {128, 256}; d_k = 128 with max_nodes <= 64 or d_k = 256 with max_nodes <= 32) and u_prev_or_null given, ONE
+ * kernel does both: the pending update is then S <- gamma_A S + sum_i (gamma_A / gamma_i) u_i k_i^T, which needs
+ * only u, k and alpha of the accepted nodes (v_prev and beta_prev are not read); outputs and the committed state
+ * carry the accuracy of that route (2e-3-grade, not fp32-grade).  On every other route -- AUTO included -- the
+ * commit and verify kernels are launched back to back on `stream`: same results at fp32 accuracy, the state
+ * crossing HBM three times.  workspace_bytes must be at least speca_workspace_bytes().
+ * After SPECA_STATUS_TIMEOUT from the one-pass kernel the state of the affected units is undefined (slices
+ * already sent back have been advanced, the others not): reload it from the caller's copy. */
 int speca_commit_verify_tree(const speca_dims *dims, float *S,
                              const uint16_t *k_prev, const uint16_t *v_prev,
                              const float *alpha_prev, const float *beta_prev,
@@ -268,7 +273,9 @@ int speca_commit_verify_tree(const speca_dims *dims, float *S,
  * other node -- and every child of the committed state -- heads a chain.  Writes chain_head[node_offsets[b]
  * + i] = local index of the first node of i's chain and n_chains[b] = the number of chains.  On any root
  * path at most floor(log2(n)) chains are entered below the first.  A sequence with bad topology is
- * reported, gets n_chains[b] = 0 and its chain_head entries are left untouched. */
+ * reported, gets n_chains[b] = 0 and its chain_head entries are left untouched.  No kernel of this library
+ * consumes the result: its own tree routes keep branch states on chip (the serial walk only borrows the
+ * heavy-path order), so the decomposition is a utility for callers that schedule chains themselves. */
 int speca_tree_mask_to_parent(int32_t batch, int32_t max_nodes, const uint8_t *mask,
                               const int32_t *node_offsets, int32_t *parent,
                               int32_t *status_word, void *stream);
@@ -315,8 +322,11 @@ int speca_commit_conv(int32_t n_layers, int32_t batch, int32_t channels, int32_t
  * Limits: dims->batch <= SPECA_NOALLOC_MAX_BATCH and total_nodes <= SPECA_NOALLOC_MAX_NODES,
  * otherwise SPECA_ERR_TOO_LARGE and nothing is launched.
  *
- * The first call on each device looks up the device address of the array (a host-side
- * query, no allocation); make that first call outside any stream capture.  Every call on
+ * The first call on each device looks up the device address of the array.  That query makes
+ * no allocation of its own, but with lazy module loading it can be the moment the CUDA runtime
+ * loads this library's device code onto that GPU (which is when the array comes to exist there):
+ * make that first call once per device during start-up, outside any stream capture and outside
+ * the latency-critical path.  The lookup may be raced by several host threads.  Every call on
  * a device uses the same array and finds in it whatever the previous call left; the
  * kernels rewrite all of it they read, so nothing needs clearing by the caller -- but two
  * calls whose kernels overlap on the GPU (different streams, no ordering between them)

@@ -1,4 +1,6 @@
 // extern "C" entry points of libspeca: argument validation and kernel dispatch only.
+#include <atomic>
+
 #include "speca_common.cuh"
 
 using namespace speca;
@@ -94,19 +96,20 @@ int verify_common(const speca_dims *dims, const float *S0, const uint16_t *q, co
 static __device__ __align__(256) unsigned char g_noalloc_scratch[SPECA_NOALLOC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-void *g_noalloc_scratch_addr[kMaxDevices] = {};
+std::atomic<void *> g_noalloc_scratch_addr[kMaxDevices];
 
-// Device address of the built-in scratch for the current device (nullptr on failure).
+// Device address of the built-in scratch for the current device (nullptr on failure).  The lookup is
+// idempotent, so two threads that race on the first call of a device store the same value.
 void *noalloc_scratch_for_current_device()
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    if (g_noalloc_scratch_addr[dev] == nullptr) {
-        void *ptr = nullptr;
+    void *ptr = g_noalloc_scratch_addr[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
-        g_noalloc_scratch_addr[dev] = ptr;
+        g_noalloc_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    return g_noalloc_scratch_addr[dev];
+    return ptr;
 }
 
 }  // namespace

@@ -42,6 +42,7 @@
 #include <cuda.h>
 
 #include <cstdlib>
+#include <mutex>
 
 #include <type_traits>
 
@@ -1389,6 +1390,50 @@ void launch_one(bool one_tile, int d_k, int grid, cudaStream_t st, const CUtenso
 
 }  // namespace
 
+namespace {
+
+struct MapKey {
+    const void *s, *q, *k, *v;
+    long units;
+    int L, T, H, DV, dk;
+    bool operator==(const MapKey &o) const
+    {
+        return s == o.s && q == o.q && k == o.k && v == o.v && units == o.units && L == o.L && T == o.T && H == o.H &&
+               DV == o.DV && dk == o.dk;
+    }
+};
+struct MapSet { CUtensorMap state; KQMaps kq; };
+// last kSets distinct (pointers, shape) keys, replaced round robin; a handful of entries, searched linearly
+class MapCache {
+public:
+    bool find(const MapKey &key, MapSet &out)
+    {
+        std::lock_guard<std::mutex> lock(mu_);
+        for (int i = 0; i < kSets; ++i)
+            if (used_[i] && keys_[i] == key) { out = sets_[i]; return true; }
+        return false;
+    }
+    void insert(const MapKey &key, const MapSet &set)
+    {
+        std::lock_guard<std::mutex> lock(mu_);
+        keys_[next_] = key; sets_[next_] = set; used_[next_] = true;
+        next_ = (next_ + 1) % kSets;
+    }
+private:
+    static constexpr int kSets = 16;
+    std::mutex mu_;
+    MapKey keys_[kSets];
+    MapSet sets_[kSets];
+    bool used_[kSets] = {};
+    int next_ = 0;
+};
+MapCache g_map_cache;
+
+int launch_with_maps(const Params &p, int d_k, bool fused, bool comp, cudaStream_t st, long n_units, const CUtensorMap &map,
+                     const KQMaps &kq);
+
+}  // namespace
+
 // Test hook of the failure-detection test (not part of the public header): with `on` the producer of CTA 0
 // never requests its first state slice, so that CTA's bounded waits run out and the call reports
 // SPECA_STATUS_TIMEOUT.  Plain (non-fused) verification only.
@@ -1402,6 +1447,11 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cu
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) return int(cudaErrorNotSupported);
     const long n_units = long(p.L) * p.B * p.H;
+    // The 13 tensor maps depend only on the four base pointers and the shape: a serving loop calls with the same
+    // ones round after round, so the last few sets are kept (a map holds addresses and strides, nothing of the data).
+    const MapKey key{p.S0, p.q, p.k, p.v, n_units, p.L, p.T, p.H, p.DV, d_k};
+    MapSet cached;
+    if (g_map_cache.find(key, cached)) return launch_with_maps(p, d_k, fused, comp, st, n_units, cached.state, cached.kq);
     CUtensorMap map;
     const int tiles = p.DV / kTileRows;
     const cuuint64_t gdim[3] = {cuuint64_t(d_k), cuuint64_t(tiles), cuuint64_t(n_units) * kTileRows};
@@ -1437,6 +1487,15 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cu
         }
     }
 
+    g_map_cache.insert(key, MapSet{map, kq});
+    return launch_with_maps(p, d_k, fused, comp, st, n_units, map, kq);
+}
+
+namespace {
+
+int launch_with_maps(const Params &p, int d_k, bool fused, bool comp, cudaStream_t st, long n_units, const CUtensorMap &map,
+                     const KQMaps &kq)
+{
     // the SM count and the opt-in to large dynamic shared memory belong to a device, not to the process
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return int(cudaErrorInvalidDevice);
@@ -1482,5 +1541,7 @@ int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cu
     else launch_one<false, false, false>(one_tile, d_k, grid, st, map, kq, fp);
     return int(cudaGetLastError());
 }
+
+}  // namespace
 
 }  // namespace speca

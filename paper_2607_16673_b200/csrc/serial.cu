@@ -139,6 +139,7 @@ verify_serial_kernel(Params p)
         int fault = 0;
         if (base < 0 || n < 0 || base + n > p.T) fault = SPECA_STATUS_BAD_OFFSETS;
         else if (n > p.max_nodes) fault = SPECA_STATUS_TOO_MANY;
+        else if (n > p.max_depth) fault = SPECA_STATUS_TOO_DEEP;      // a chain of n nodes is n levels deep, on every route
         if (fault) {
             if (threadIdx.x == 0 && blockIdx.x % tiles == 0 && h == 0 && l == 0) atomicOr(p.status, fault);
             return;

@@ -592,3 +592,18 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
     dp.verify_tree()
     assert dp.status_value() == 0
     assert rel_err(cpu(dp.o), oracle_verify(prob)) <= TOL_FP32
+
+
+@pytest.mark.parametrize("route", [speca.ROUTE_SERIAL, speca.ROUTE_AUTO])
+def test_chain_longer_than_max_depth_is_a_fault_on_every_route(route):
+    """A chain of n nodes is n levels deep: the chain entry point reports TOO_DEEP and skips the sequence whatever
+    kernel verifies it."""
+    prob = synth.make_problem(1400, 1, 2, 128, 128, [synth.chain_parent(6), synth.chain_parent(12)], max_depth=16)
+    good = oracle_verify(prob)
+    dp = DevProblem(prob, route=route, max_nodes=16)
+    dp.dims.max_depth = 8
+    dp.verify_chain()
+    assert dp.status_value() == speca.STATUS_TOO_DEEP
+    o = cpu(dp.o)
+    assert np.all(np.isnan(o[:, 6:]))
+    assert rel_err(o[:, :6], good[:, :6]) <= TOL_FP32

@@ -76,3 +76,38 @@ def test_algorithmic_bytes_formula():
     units, Sb = L * B * H, 4 * dk * dv
     assert v == units * Sb + T * L * H * (4 * dk + 2 * dv + 8) + T * L * H * 4 * dv == 10080485376
     assert c == 2 * 100 * L * H * Sb + 200 * L * H * (2 * dk + 2 * dv + 8)
+
+
+def test_gpus_flag_starts_one_rank_per_gpu(monkeypatch):
+    """`python bench.py --gpus N` outside a launcher re-executes itself under torch.distributed.run with N ranks on
+    127.0.0.1; inside a launcher (WORLD_SIZE set) it must not spawn again."""
+    calls = []
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: calls.append(cmd) or 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "1"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 0 and len(calls) == 1
+    cmd = calls[0]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "2", "--steps", "1"] and os.path.basename(cmd[-5]) == "bench.py"
+
+
+def test_launcher_runs_two_ranks_end_to_end_on_cpu():
+    """The same launch line the multi-GPU benchmark uses, with the arm that needs no GPU: two ranks start, rank 0
+    prints the one JSON line, rank 1 exits 0 without output."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                        "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"),
+                        "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "1"],
+                       env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2

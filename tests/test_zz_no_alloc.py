@@ -6,7 +6,7 @@ a latency-critical stream that must never hit the device-wide synchronisation of
 cudaMalloc.  For them the library carries its own fixed scratch array.  This test calls
 that entry point through the C ABI twice in a row (the second call finds the first
 call's leftovers in the array) and checks both results against the ordinary entry point
-fed with a caller-allocated workspace.
+fed with a caller-allocated workspace, and against the fp64 oracle.
 
 Collected last on purpose, so that a run stopping at the first failure has already run
 every other test; it must also pass alone in a fresh process.
@@ -19,7 +19,7 @@ import torch
 
 from paper_2607_16673_b200 import binding as speca
 from paper_2607_16673_b200 import synth
-from gpu_util import DevProblem, TOL_FP32, rel_err
+from gpu_util import DevProblem, TOL_FP32, oracle_verify, rel_err
 
 
 def _problem(seed, sizes):
@@ -46,6 +46,8 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(route):
         assert rel_err(dp.o.cpu().numpy(), ref.o.cpu().numpy()) <= TOL_FP32
         assert rel_err(dp.u.cpu().numpy(), ref.u.cpu().numpy()) <= TOL_FP32
         assert torch.equal(dp.S, ref.S)
+        # and an error common to both entry points would show against the oracle
+        assert rel_err(dp.o.cpu().numpy(), oracle_verify(prob)) <= TOL_FP32
 
 
 @pytest.mark.gpu
