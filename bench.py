@@ -453,7 +453,8 @@ def run_speca(args):
                              3: "single-pass TF32", 4: "effective-query"}.get(args.route, str(args.route)),
                    "parallelism": f"dp{world} (sequences partitioned, no collective)"},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic(args.workload, dom) if not args.layers and not args.batch else None,
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": (ncu_traffic(args.workload + {3: "-tf32", 4: "-effective"}.get(args.route, "") if dom == "verify" else args.workload, dom)
+                                 if not args.layers and not args.batch else None),
                      "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms},
         "kernels": {"verify_ms": t_verify, "accept_ms": t_accept, "commit_ms": t_commit,
                     "verify_single_pass_tf32_ms": tf32_ms,
@@ -558,8 +559,11 @@ def ncu_traffic(workload: str, kernel: str):
             for line in f:
                 cells = [c.strip() for c in line.strip().strip("|").split("|")]
                 if len(cells) >= 4 and cells[0] == workload and cells[1] == kernel:
-                    return float(cells[2]) * float(cells[3])
-    except (OSError, ValueError):
+                    try:
+                        return float(cells[2]) * float(cells[3])
+                    except ValueError:
+                        continue
+    except OSError:
         pass
     return None
 

@@ -76,7 +76,12 @@ constexpr int kThreads = 14 * 32;
 constexpr int kUpdWarps = 2;                   // state-update role of the fused kernel
 constexpr int kUpdThreads = kUpdWarps * 32;
 constexpr int kThreadsFused = kThreads + kUpdThreads;
-constexpr int kThreadsComp = kThreads + 5 * 32;  // compensated form: a second MMA issuer and four warps that rewrite slices
+#ifndef SPECA_SPLIT_WARPS
+#define SPECA_SPLIT_WARPS 4
+#endif
+constexpr int kSplitWarps = SPECA_SPLIT_WARPS;      // warps that rewrite slices as their remainder
+constexpr int kSplitThreads = kSplitWarps * 32;
+constexpr int kThreadsComp = kThreads + (1 + kSplitWarps) * 32;  // compensated form: a second MMA issuer and the split warps
 constexpr int kPrepThreads = 128;
 // The tensor core reads an fp32 state element as TF32 by dropping its low 13 mantissa bits, i.e. it
 // rounds every element toward zero: on average a value with mantissa m in [1, 2) loses 2^-11 / m of
@@ -419,7 +424,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
             mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarUpd + s), kUpdThreads);
             mbar_init(bar(kBarP1Done + s), 1);
-            mbar_init(bar(kBarLo + s), 4);
+            mbar_init(bar(kBarLo + s), kSplitWarps);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(kBarPendFull + i), 1); mbar_init(bar(kBarPendFree + i), kUpdThreads); }
         mbar_init(bar(kBarBReady), kPrepThreads);
@@ -755,10 +760,10 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 // the remainders are formed while the first pass is still reading the slice; only the stores wait
                 if (!(ok = WAIT(0, bar(kBarFull + s), ph))) break;
                 float4 *sl = reinterpret_cast<float4 *>(smem + kOffRing + s * kStageBytes);
-                float4 v[kStageBytes / 16 / 128];
+                float4 v[kStageBytes / 16 / kSplitThreads];
 #pragma unroll
-                for (int k = 0; k < kStageBytes / 16 / 128; ++k) {
-                    v[k] = sl[stid + k * 128];
+                for (int k = 0; k < kStageBytes / 16 / kSplitThreads; ++k) {
+                    v[k] = sl[stid + k * kSplitThreads];
                     v[k].x -= __uint_as_float(__float_as_uint(v[k].x) & 0xffffe000u);
                     v[k].y -= __uint_as_float(__float_as_uint(v[k].y) & 0xffffe000u);
                     v[k].z -= __uint_as_float(__float_as_uint(v[k].z) & 0xffffe000u);
@@ -766,7 +771,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                 }
                 if (!(ok = WAIT(1, bar(kBarP1Done + s), ph))) break;
 #pragma unroll
-                for (int k = 0; k < kStageBytes / 16 / 128; ++k) sl[stid + k * 128] = v[k];
+                for (int k = 0; k < kStageBytes / 16 / kSplitThreads; ++k) sl[stid + k * kSplitThreads] = v[k];
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarLo + s));
