@@ -19,26 +19,33 @@
 // Accuracy.  The tensor core reads fp32 operands as TF32 (top 19 bits).  Both operands are
 // therefore split: the state slice as landed (its TF32 head, free) and its exact remainder
 // S - tf32(S), rewritten in place by a CUDA-core role once the first pass has read the slice;
-// the effective vectors as a TF32-rounded head and the exact remainder, stacked as 2R operand
-// rows.  Pass 1: S x [head; tail] -> accumulator columns [0,R) and [R,2R); pass 2: (S - tf32(S)) x
-// head -> columns [0,R).  The dropped term is 2^-22 of the result.  Mq / Mk are split into three
-// bf16 pieces (24 bits) and multiply the bf16 value rows exactly.
+// the effective vectors as a TF32-rounded head and the exact remainder.  First pass: S x head ->
+// accumulator columns [0,R); correction passes: S x tail and then (S - tf32(S)) x head -> columns
+// [R,2R).  The dropped term is 2^-22 of the result.  Mq / Mk are split into three bf16 pieces
+// (24 bits) and multiply the bf16 value rows exactly.
 //
-// Mapping.  One persistent CTA per SM walks units (layer, sequence, head); 19 warps:
-//   warp 0       TMA producer: per unit the K-slices of the fp32 state (128-byte swizzle), slice by slice
-//                over both value tiles, and, after the first slice pair, the unit's bf16 value rows --
-//                all through one ring of 16 KiB slots;
-//   warps 1, 18  issue the tcgen05.mma of value tile 0 / 1 (an instruction costs its issuer about a
-//                hundred cycles and a unit needs about a hundred of them); warp 1 owns TMEM (two
-//                units of accumulators in flight) and issues the Gram blocks;
-//   warps 2-5    solver: ancestor entries of the Gram block out of TMEM, the two back substitutions,
-//                one record per operand row, the three bf16 pieces of M -- one unit ahead;
-//   warps 6-9    effective vectors from the records and the staged bf16 keys / queries, one K-slice
-//                at a time into a double-buffered operand (so they never exist whole);
-//   warps 10-13  rewrite each state slice as its TF32 remainder between the two passes;
-//   warps 14-17  epilogue: o (or u) = column t + column R + t, streamed out coalesced.
+// Mapping.  One persistent CTA per SM walks units (layer, sequence, head); 21 warps:
+//   warp 0        TMA producer: per unit the K-slices of the fp32 state (128-byte swizzle), slice by slice
+//                 over both value tiles, and, after the first slice pair, the unit's bf16 value rows --
+//                 all through one ring of 16 KiB slots;
+//   warps 1, 18   issue the first-pass tcgen05.mma of value tile 0 / 1 and the value-row product (an
+//                 instruction costs its issuer about 130 cycles and a unit needs about a hundred of
+//                 them, hence several issuers); warp 1 owns TMEM (two units of accumulators in flight)
+//                 and issues the Gram blocks;
+//   warps 19, 20  issue the correction passes of tile 0 / 1, each following two cursors (the tail
+//                 operand, ready as soon as the slice has landed; the rewritten slice, ready once the
+//                 split role is done with it) and releasing the ring slot;
+//   warps 2-5     solver: ancestor entries of the Gram block out of TMEM, the two back substitutions,
+//                 one record per operand row, the three bf16 pieces of M -- one unit ahead;
+//   warps 6-9     effective vectors from the records and the staged bf16 keys / queries, one K-slice
+//                 at a time into a ring of operand slices (so they never exist whole);
+//   warps 10-13   rewrite each state slice as its TF32 remainder between the passes;
+//   warps 14-17   epilogue: o (or u) = column t + column R + t, streamed out coalesced.
+// Every visit of a ring slot, state slice or value rows, completes the same four barriers in the
+// same order (landed, first pass read, rewritten, released), so that their phase parities stay in step.
 // Nodes keep their index order everywhere.  When u is requested a unit is walked twice (first the
-// o rows, then the u rows); the second walk finds the state tile in L2.
+// o rows, then the u rows); the second walk finds the state tile in L2.  The order in which the
+// passes reach an accumulator column is not fixed, so two runs may differ in the last bit.
 // Every wait is bounded; on expiry the CTA raises SPECA_STATUS_TIMEOUT, drains and exits.
 #include <cuda.h>
 
@@ -174,13 +181,6 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
 
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-// two fp32 -> packed bf16 pair (round to nearest even), low half first
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 // what the tensor core's TF32 reading of x (low 13 mantissa bits dropped) leaves out; exact
 __device__ __forceinline__ float tf32_rest(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16])

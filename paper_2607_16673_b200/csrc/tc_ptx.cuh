@@ -225,10 +225,11 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
         : "memory");
 }
 
-// K-major operand, 128-byte swizzle (the descriptor above), for operands whose MN extent is contiguous
-// instead: rows of 128 bytes hold 64 consecutive 16-bit MN elements of one K index, 8 K indices form a
-// 1024-byte group (stride byte offset), the next 64 MN elements start `mn_block_bytes` further (leading
-// byte offset).
+// MN-major operand with the 128-byte swizzle: the operand sits in shared memory with its M (or N) extent
+// contiguous, as a row-major [K][MN] tile of 16-bit elements.  A row of 128 bytes holds 64 consecutive MN
+// elements of one K index, 8 K indices form a 1024-byte group (stride byte offset), and the next 64 MN
+// elements start `mn_block_bytes` further on (leading byte offset).  The instruction descriptor must mark
+// the operand as MN-major (make_idesc_bf16_amn).
 __device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr, uint32_t mn_block_bytes)
 {
     uint64_t d = 0;

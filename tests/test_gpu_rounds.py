@@ -10,7 +10,7 @@ import torch
 import oracle
 from paper_2607_16673_b200 import binding as speca
 from paper_2607_16673_b200 import synth
-from gpu_util import TOL, TOL_FP32, rel_err
+from gpu_util import TOL, TOL_FP32, max_err_over_max, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -55,7 +55,7 @@ def run_rounds(kind, L, B, rounds, route, tol, n_sample=24, seed=77):
     path_idx = torch.zeros(B, 8, dtype=torch.int32, device="cuda")
     path_len = torch.zeros(B, dtype=torch.int32, device="cuda")
     next_tok = torch.zeros(B, dtype=torch.int32, device="cuda")
-    worst_o = worst_s = 0.0
+    worst_o = worst_s = mom_o = mom_s = 0.0
     accepted = []
     for r in range(rounds):
         parents, offs, parent, depth, draft, target, root = host_topology(kind, B, seed + 100 + r)
@@ -79,15 +79,17 @@ def run_rounds(kind, L, B, rounds, route, tol, n_sample=24, seed=77):
         o_gpu = np.concatenate([o[l, int(offs[b]):int(offs[b + 1]), h].cpu().numpy() for (l, b, h) in units])
         assert not np.isnan(o_gpu).any()
         worst_o = max(worst_o, rel_err(o_gpu, o_ref[0, :, 0]))
+        mom_o = max(mom_o, max_err_over_max(o_gpu, o_ref[0, :, 0]))
         speca.commit(dims, S, k, v, al, be, d_offs, T, d_par, path_idx, path_len, status)
         sub_pi = np.stack([pi[b] for (_, b, _) in units]); sub_pl = np.asarray([pl[b] for (_, b, _) in units], np.int32)
         S_ref = oracle.commit(sp["S"], sp["k"], sp["v"], sp["alpha"], sp["beta"], sp["offs"], sub_pi, sub_pl)[0, :, 0]
         S_gpu = np.stack([S[l, b, h].cpu().numpy() for (l, b, h) in units])
         worst_s = max(worst_s, rel_err(S_gpu, S_ref))
+        mom_s = max(mom_s, max_err_over_max(S_gpu, S_ref))
         accepted.append(float(pl.mean()))
         assert int(status.item()) == 0
-    print(f"{kind} route={route} rounds={rounds}: worst verify err {worst_o:.3e}, worst state err {worst_s:.3e}, "
-          f"mean accepted {np.mean(accepted):.2f}")
+    print(f"{kind} route={route} rounds={rounds}: worst verify err {worst_o:.3e} (max|x-r|/max|r| {mom_o:.3e}), "
+          f"worst state err {worst_s:.3e} (max|x-r|/max|r| {mom_s:.3e}), mean accepted {np.mean(accepted):.2f}")
     assert worst_o <= tol and worst_s <= TOL_FP32 * 4
     return worst_o, worst_s
 
@@ -133,7 +135,7 @@ def run_rounds_fused(kind, L, B, rounds, tol, n_sample=24, seed=177, H=16, dk=12
              for _ in range(2)]
     next_tok = torch.zeros(B, dtype=torch.int32, device="cuda")
     t = lambda a: torch.from_numpy(a).cuda()
-    worst_o = worst_s = 0.0
+    worst_o = worst_s = mom_o = mom_s = 0.0
     prev = prev_host = None
     for r in range(rounds + 1):
         flush = r == rounds
@@ -171,6 +173,7 @@ def run_rounds_fused(kind, L, B, rounds, tol, n_sample=24, seed=177, H=16, dk=12
         assert int(status.item()) == 0
         S_gpu = np.stack([S[l, b, h].cpu().numpy() for (l, b, h) in units])
         worst_s = max(worst_s, rel_err(S_gpu, S_ref))
+        mom_s = max(mom_s, max_err_over_max(S_gpu, S_ref))
         if flush:
             break
         sp = sample_problem(units, parents, offs, S_ref, q, k, v, al, be, dk, dv)
@@ -180,9 +183,11 @@ def run_rounds_fused(kind, L, B, rounds, tol, n_sample=24, seed=177, H=16, dk=12
         o_gpu = np.concatenate([o[l, int(offs[b]):int(offs[b + 1]), h].cpu().numpy() for (l, b, h) in units])
         assert not np.isnan(o_gpu).any()
         worst_o = max(worst_o, rel_err(o_gpu, o_ref[0, :, 0]))
+        mom_o = max(mom_o, max_err_over_max(o_gpu, o_ref[0, :, 0]))
         prev = dict(k=k, v=v, alpha=al, beta=be, u=u, node_offsets=d_offs, total_nodes=T, parent=d_par)
         prev_host = (sp, np.stack([pi[b] for (_, b, _) in units]), np.asarray([pl[b] for (_, b, _) in units], np.int32))
-    print(f"fused {kind} L={L} B={B} rounds={rounds}: worst verify err {worst_o:.3e}, worst state err {worst_s:.3e}")
+    print(f"fused {kind} L={L} B={B} rounds={rounds}: worst verify err {worst_o:.3e} (max|x-r|/max|r| {mom_o:.3e}), "
+          f"worst state err {worst_s:.3e} (max|x-r|/max|r| {mom_s:.3e})")
     assert worst_o <= tol and worst_s <= tol
     return worst_o, worst_s
 
