@@ -1018,7 +1018,7 @@ def run_sweep(args):
         q, k, v, al, be = synth.device_records(7, L, hi["T"], H, dk, dv, dev)
         dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, args.route)
         offs, par = t(hi["node_offsets"]), t(hi["parent"])
-        for A in (1, 2, 4, 8):
+        for A in (1, 2, 3, 4, 5, 6, 8):
             pidx = torch.arange(8, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()
             plen = torch.full((B,), A, dtype=torch.int32, device=dev)
             ms = timed(lambda: speca.commit(dims, S, k, v, al, be, offs, hi["T"], par, pidx, plen, status))

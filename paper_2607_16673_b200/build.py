@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspeca.so")
-SOURCES = ["api.cu", "plan.cu", "serial.cu", "factorized.cu", "effective.cu"]
+SOURCES = ["api.cu", "plan.cu", "serial.cu", "commit_mma.cu", "factorized.cu", "effective.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

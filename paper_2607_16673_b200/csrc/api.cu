@@ -127,6 +127,11 @@ void speca_test_withhold_first_load(int on)
     effective_set_withhold(on);
 }
 
+/* Test hook, deliberately absent from speca.h: speca_commit hands accepted paths of four to eight nodes to its
+ * tensor-core kernel only when the batch is large enough for throughput to matter (n 16-row tiles per resident
+ * warp; default 128).  n = 0 makes every batch of a supported shape take it, n < 0 restores the default. */
+void speca_test_commit_long_min_tiles(int n) { commit_long_set_min_tiles_per_warp(n); }
+
 const char *speca_strerror(int code)
 {
     switch (code) {

@@ -220,6 +220,8 @@ commit_kernel(Params p)
     const int base = __ldg(p.node_offsets + b);
     const int n = __ldg(p.node_offsets + b + 1) - base;
     if (len == 0) return;
+    // paths the tensor-core commit takes (it validates them itself)
+    if (p.long_min > 0 && len >= p.long_min && len <= 8 && len <= p.max_depth) return;
 
     // Start streaming the state tile right away; the accepted path is validated in the
     // shadow of these loads (one thread per path step), and nothing is stored if it is bad.
@@ -391,8 +393,18 @@ int launch_decode(const Params &p, int d_k, cudaStream_t st)
     return int(cudaErrorInvalidValue);
 }
 
-int launch_commit(const Params &p, int d_k, cudaStream_t st)
+// Accepted paths of kCommitLongMin nodes or more go to the tensor-core kernel where it takes the shape: from there
+// on the token-by-token form is bound by its arithmetic, not by HBM.
+constexpr int kCommitLongMin = 4;
+
+int launch_commit(const Params &p_in, int d_k, cudaStream_t st)
 {
+    Params p = p_in;
+    p.long_min = (p.max_depth >= kCommitLongMin && commit_long_supported(p, d_k)) ? kCommitLongMin : 0;
+    if (p.long_min > 0) {
+        const int rc = launch_commit_long(p, d_k, st);
+        if (rc != 0) return rc;
+    }
     switch (d_k) {
     case 64: return pick_tile<64, LaunchCommit>(p, st);
     case 128: return pick_tile<128, LaunchCommit>(p, st);

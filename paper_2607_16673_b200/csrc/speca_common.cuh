@@ -91,6 +91,7 @@ struct Params {
     int32_t *status;
     Workspace ws;
     int32_t n_slots;             // on-chip state slots available to the tree walk
+    int32_t long_min;            // commit: accepted paths of long_min..8 nodes are taken by the tensor-core kernel (0: none)
 };
 
 // Launchers implemented per translation unit; each returns a cudaError_t-compatible int.
@@ -98,6 +99,10 @@ int launch_plan(const Params &p, cudaStream_t st);
 int launch_decode(const Params &p, int d_k, cudaStream_t st);
 int launch_verify_serial(const Params &p, int d_k, bool chain, cudaStream_t st);
 int launch_commit(const Params &p, int d_k, cudaStream_t st);
+// commit of paths of p.long_min..8 nodes on warp-level MMAs (the token-by-token kernel skips those sequences)
+bool commit_long_supported(const Params &p, int d_k);
+int launch_commit_long(const Params &p, int d_k, cudaStream_t st);
+void commit_long_set_min_tiles_per_warp(int n);
 bool factorized_supported(const speca_dims *d);
 bool factorized_fused_supported(const speca_dims *d);
 int launch_verify_factorized(const Params &p, int d_k, bool fused, bool comp, cudaStream_t st);
