@@ -465,7 +465,9 @@ def run_speca(args):
         "decode_step": {"ms": dec_ms, "gbs": dec_bytes / (dec_ms * 1e-3) / 1e9,
                         "token_layers_per_s": B * L / (dec_ms * 1e-3),
                         "note": "one autoregressive token per sequence at the same batch"},
-        "gpu_launches": 4 * K,
+        # plan, verify, accept, commit -- and the long-path commit kernel in front of it where the batch is large enough
+        # for the library to use it (d_k <= 128, at least 128 16-row tiles per resident warp; 16 warps per SM)
+        "gpu_launches": (5 if dk <= 128 and L * B * H * (dv // 16) >= 128 * 16 * torch.cuda.get_device_properties(dev).multi_processor_count else 4) * K,
         "conv_commit": {"ms": conv_ms, "channels": ch, "width": W, "gbs": conv_bytes / (conv_ms * 1e-3) / 1e9,
                         "note": "speca_commit_conv on the accepted paths of one round; outside the timed step"},
         "draft_utils": {"tree_mask_to_parent_ms": mask_ms, "prune_tree_ms": prune_ms, "stochastic_accept_ms": sacc_ms, "chain_decompose_ms": chain_ms,

@@ -191,10 +191,17 @@ int speca_stochastic_accept(int32_t batch, int32_t max_depth,
 
 /* Commit (Section 5.1 factor buffering, Eq. 3; Section 5.2 immediate update): gathers
  * the factor records (k, v, alpha, beta) on the accepted path path_idx[b][0..path_len[b])
- * and advances S over them in place, token by token, in fp32.  path_len[b] == 0 leaves
+ * and advances S over them in place, in fp32.  path_len[b] == 0 leaves
  * the sequence's state bitwise untouched (it is neither read nor written).  If
  * parent_or_null is given the path is checked to be a chain of parent links starting at
- * a child of the committed state; an invalid path skips the sequence. */
+ * a child of the committed state; an invalid path skips the sequence.
+ * The state is advanced token by token; in large batches (d_k <= 128) paths of four to
+ * eight nodes are advanced in the unrolled form of Section 4.2 instead (one product of the
+ * state tile with all keys of the path, the recurrence per row, one rank-A update, on
+ * tensor cores with every fp32 operand split into a TF32 head and its exact remainder).
+ * Both forms carry fp32 accuracy; they differ in rounding order, so the state of a
+ * sequence is reproducible for a given batch shape, not across batch shapes.  The call
+ * launches one or two kernels on `stream`. */
 int speca_commit(const speca_dims *dims, float *S,
                  const uint16_t *k, const uint16_t *v,
                  const float *alpha, const float *beta,
