@@ -59,7 +59,7 @@ def parse_args():
     ap.add_argument("--impl", default="speca", choices=["speca", "reference"])
     ap.add_argument("--route", type=int, default=0,
                     help="0 auto (fp32-grade), 1 serial, 2 factorised (fp32-grade), 3 single-pass TF32, 4 effective-query")
-    ap.add_argument("--sweep", default=None, choices=["commit-len", "unit-types"],
+    ap.add_argument("--sweep", default=None, choices=["commit-len", "unit-types", "role-waits"],
                     help="commit-len: commit throughput against the accepted path length; unit-types: time per "
                          "(layer, sequence, head) unit and SM of 8-token chains and 64-node trees, per route")
     ap.add_argument("--e2e-steps", type=int, default=6)
@@ -1026,6 +1026,39 @@ def run_sweep(args):
             ms = timed(lambda: speca.commit(dims, S, k, v, al, be, offs, hi["T"], par, pidx, plen, status))
             nbytes = 2 * L * B * H * 4 * dk * dv + A * B * L * H * (2 * dk + 2 * dv + 8)
             rows.append({"accepted": A, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peak})
+    elif args.sweep == "role-waits":
+        # Per-role wait cycles of the tensor-core verification, recorded by CTA 0 of a library built with -DSPECA_PROF
+        # (SPECA_NVCC_FLAGS=-DSPECA_PROF python -m paper_2607_16673_b200.build --force): for one warp of every role its
+        # lifetime in cycles and the share of it spent in each of up to eight kinds of wait or code segment (the slot
+        # numbers are the first argument of the WAIT / PROF_SEG macros in the kernel source).  The instrumented build
+        # is 20-40 % slower than the plain one: read the shares, not the times.
+        if not speca.lib().speca_test_profiling_build():
+            print(json.dumps({"sweep": args.sweep, "error": "library not built with -DSPECA_PROF: rebuild with "
+                              "SPECA_NVCC_FLAGS=-DSPECA_PROF python -m paper_2607_16673_b200.build --force"}))
+            return
+        L = args.layers or 4
+        S = synth.device_state(1, L, B, H, dk, dv, 0.02, dev)
+        roles = {0: {0: "TMA producer", 1: "MMA issuer, tile 0", 14: "MMA issuer, tile 1", 2: "preparation", 6: "epilogue group 0",
+                     10: "epilogue group 1", 15: "split"},
+                 3: {0: "TMA producer", 1: "MMA issuer", 2: "preparation", 6: "epilogue group 0", 10: "epilogue group 1"},
+                 4: {0: "TMA producer", 1: "first pass, tile 0", 18: "first pass, tile 1", 19: "correction, tile 0",
+                     20: "correction, tile 1", 2: "solver", 6: "vector", 10: "split", 14: "epilogue"}}
+        sm = torch.cuda.get_device_properties(dev).multi_processor_count
+        for wl in ("chains8", "trees64", "cfg5"):
+            hi = host_round_inputs(wl, B, 5000)
+            q, k, v, al, be = synth.device_records(7, L, hi["T"], H, dk, dv, dev)
+            offs, par = t(hi["node_offsets"]), t(hi["parent"])
+            o = torch.empty(L, hi["T"], H, dv, device=dev)
+            dims = speca.Dims(L, B, H, dk, dv, 1.0, 8, 64, args.route)
+            ws = speca.alloc_workspace(dims, hi["T"], dev)
+            ms = timed(lambda: speca.verify_tree(dims, S, q, k, v, al, be, offs, hi["T"], par, None, o, None, ws, status), reps=1)
+            ctrl = ws[:2048].cpu().numpy().view(np.int64)
+            for w, name in roles.get(args.route, roles[0]).items():
+                vals = ctrl[8 + w * 9: 8 + w * 9 + 9]
+                if vals[8] > 0:
+                    rows.append({"units": wl, "warp": w, "role": name, "life_kcycles": float(vals[8]) / 1e3,
+                                 "share_pct": [round(100.0 * float(x) / float(vals[8]), 1) for x in vals[:8]]})
+            rows.append({"units": wl, "verify_ms": ms, "us_per_unit_per_sm": ms * 1e3 / (L * B * H / sm)})
     else:
         sm = torch.cuda.get_device_properties(dev).multi_processor_count
         for wl in ("chains8", "trees64"):

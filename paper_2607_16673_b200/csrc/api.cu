@@ -132,6 +132,18 @@ void speca_test_withhold_first_load(int on)
  * warp; default 128).  n = 0 makes every batch of a supported shape take it, n < 0 restores the default. */
 void speca_test_commit_long_min_tiles(int n) { commit_long_set_min_tiles_per_warp(n); }
 
+/* Not in speca.h: 1 if the library was compiled with -DSPECA_PROF (the tensor-core kernels then record, for CTA 0,
+ * the cycles each role spends in each kind of wait at the start of the workspace; bench.py --sweep role-waits
+ * reads them). */
+int speca_test_profiling_build(void)
+{
+#ifdef SPECA_PROF
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 const char *speca_strerror(int code)
 {
     switch (code) {
