@@ -250,7 +250,13 @@ __device__ __forceinline__ bool next_unit(const UnitWalk &w, Unit &x)
 // branch-free.  The u of the nodes on the current depth-first path live in ustk[.][depth-1];
 // coefficients of levels that are not ancestors of this node are zero.
 //   cf[0..6] cU   cf[7] cV   cf[8..15] cO   cf[16] cR   cf[17] cG   cf[18] depth-1   cf[19] output offset
-template <int TP>
+// SELF: the coefficient of the node's own u (q.k) sits in cO[7] whatever the depth and the last stack slot always
+// takes the node's own u (a node at depth 8 has no children, so that slot is never an ancestor's): one select and one
+// compare fewer per row, and a leaf can stay out of the stack altogether (level -1 in its record), so that the sums
+// of the node after it do not depend on it (64-node trees 10.8 -> 10.5 us per unit in the compensated kernel, 9.4 ->
+// 9.15 in the single-pass one).  A form of the step on packed two-wide fp32 FMAs was measured equal on trees, 1.5 %
+// better on 8-node chains and spills at the compensated kernel's 96 registers; it is not kept.
+template <int TP, bool SELF = false>
 __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const float *cf, const float (&Rv)[TP],
                                           const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
                                           float (&o_out)[TP], int &off)
@@ -272,7 +278,8 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
         u0 = fmaf(a1.z, ustk[t][6], u0);
         const float u = u0 + u1;
 #pragma unroll
-        for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        for (int j = 0; j < kMaxDepth - (SELF ? 1 : 0); ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        if (SELF) ustk[t][kMaxDepth - 1] = u;
         float o0 = fmaf(b0.x, ustk[t][0], s.y * Gv[t]);
         float o1 = b0.y * ustk[t][1];
         o0 = fmaf(b0.z, ustk[t][2], o0);
@@ -282,68 +289,6 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
         o0 = fmaf(b1.z, ustk[t][6], o0);
         o1 = fmaf(b1.w, ustk[t][7], o1);
         o_out[t] = o0 + o1;
-        u_out[t] = u;
-    }
-}
-
-// packed fp32 pairs (sm_100: two IEEE operations per instruction)
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c)
-{
-    unsigned long long d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b)
-{
-    unsigned long long d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-
-// The 8-level step with the levels taken two at a time by packed fp32 FMAs (each half an IEEE
-// fma): the pairs (cU[2i], cU[2i+1]) come out of the 128-bit loads as they are, and the stack is
-// read as the matching pairs of levels.  Level 7 is never an ancestor (a node has at most 7), so
-// its slot carries v through the u step, paired with cV, and the node's own u afterwards if the
-// node is at depth 8; cO[7] is zero otherwise.  Used by the plain kernel (it is no gain in the
-// fused one, whose update role competes for the same issue slots).
-template <int TP>
-__device__ __forceinline__ void node_step_packed(float (&ustk)[TP][kMaxDepth], const float *cf, const float (&Rv)[TP],
-                                                 const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
-                                                 float (&o_out)[TP], int &off)
-{
-    const ulonglong2 a0 = *reinterpret_cast<const ulonglong2 *>(cf + 0), a1 = *reinterpret_cast<const ulonglong2 *>(cf + 4);
-    const ulonglong2 b0 = *reinterpret_cast<const ulonglong2 *>(cf + 8), b1 = *reinterpret_cast<const ulonglong2 *>(cf + 12);
-    const float4 s = *reinterpret_cast<const float4 *>(cf + 16);
-    const int d1 = __float_as_int(s.z);
-    off = __float_as_int(s.w);
-#pragma unroll
-    for (int t = 0; t < TP; ++t) {
-        ustk[t][7] = vv[t];
-        unsigned long long acc = mul2(a0.x, pack2(ustk[t][0], ustk[t][1]));
-        acc = fma2(a0.y, pack2(ustk[t][2], ustk[t][3]), acc);
-        acc = fma2(a1.x, pack2(ustk[t][4], ustk[t][5]), acc);
-        acc = fma2(a1.y, pack2(ustk[t][6], ustk[t][7]), acc);
-        float e, f;
-        unpack2(acc, e, f);
-        const float u = fmaf(s.x, Rv[t], e + f);
-#pragma unroll
-        for (int j = 0; j < kMaxDepth; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
-        acc = mul2(b0.x, pack2(ustk[t][0], ustk[t][1]));
-        acc = fma2(b0.y, pack2(ustk[t][2], ustk[t][3]), acc);
-        acc = fma2(b1.x, pack2(ustk[t][4], ustk[t][5]), acc);
-        acc = fma2(b1.y, pack2(ustk[t][6], ustk[t][7]), acc);
-        unpack2(acc, e, f);
-        o_out[t] = fmaf(s.y, Gv[t], e + f);
         u_out[t] = u;
     }
 }
@@ -461,6 +406,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int NS = FUSED ? kStagesFused : kStages;            // ring depth in use
+    constexpr bool kSelfSlot = !DEEP;                             // see node_step
     static_assert(DK == 128 || DK == 256, "key width");
     constexpr int NC = DK / kChunkK;                              // K-chunks (state slices) per tile
     constexpr int BROWS = DK == 128 ? kBopRows : kBopRows / 2;    // [K;Q] rows the operand buffers hold
@@ -1033,16 +979,18 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                         reinterpret_cast<float4 *>(cf)[i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
                     cf[2 * MAXD] = (active && !p.no_erase) ? sgn * ratio * (COMP ? 1.f : kDebias) : 0.f;      // cR = -beta gamma
                 } else {
-                    // level d-1 is the node itself: (q_t . k_t) with ratio 1
+                    // level d-1 is the node itself: (q_t . k_t) with ratio 1 (kSelfSlot: kept in the last slot)
                     c[MAXD - 1] = 0.f;
 #pragma unroll
                     for (int j = 0; j < MAXD; ++j)
-                        if (active && j == d - 1) c[j] = sgn * gsel[j];
+                        if (active && j == d - 1) c[kSelfSlot ? MAXD - 1 : j] = sgn * gsel[j];
 #pragma unroll
                     for (int i = 0; i < MAXD / 4; ++i)
                         reinterpret_cast<float4 *>(cf)[MAXD / 4 + i] = make_float4(c[4 * i], c[4 * i + 1], c[4 * i + 2], c[4 * i + 3]);
                     cf[2 * MAXD + 1] = active ? sgn * ratio * (COMP ? 1.f : kDebias) : 0.f;                  // cG = scale gamma
-                    cf[2 * MAXD + 2] = __int_as_float(active ? d - 1 : -1);
+                    // (kSelfSlot: a leaf's u is nobody's ancestor term -- level -1 keeps it out of the stack, so that the
+                    // next node's sums do not wait for it)
+                    cf[2 * MAXD + 2] = __int_as_float((active && !(kSelfSlot && ((meta.x >> 16) & 1))) ? d - 1 : -1);
                     cf[2 * MAXD + 3] = __int_as_float(active ? node * p.H * p.DV : 0);        // offset of the node's row
                 }
             }
@@ -1153,8 +1101,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                         v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
                     }
                     if constexpr (DEEP) node_step_deep<TP, MAXD>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
-                    else if constexpr (FUSED) node_step<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
-                    else node_step_packed<TP>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
+                    else node_step<TP, kSelfSlot>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
                     if (p0 + i < n) {
                         if (TP == 2) {
                             *reinterpret_cast<float2 *>(o_row + off) = make_float2(oo[0], oo[TP - 1]);

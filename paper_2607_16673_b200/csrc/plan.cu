@@ -111,7 +111,7 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
         posn[i] = pos;
     }
     __syncthreads();
-    // Per node: depth, position in the processing order, and the node's ancestors by depth
+    // Per node: depth, position in the processing order, a leaf flag, and the node's ancestors by depth
     // (one byte each; meaningful for sequences of <= 256 nodes and depth <= 16, which is all
     // the factorised route accepts).  Level j (0 = child of the committed state) of the first
     // record sits in byte j % 4 of word 1 + j / 4 for j < 12; levels 12..14 are in the second.
@@ -125,7 +125,7 @@ plan_kernel(const int32_t *__restrict__ node_offsets, const int32_t *__restrict_
             if (j < 16) w[j >> 2] |= (uint32_t(a) & 0xffu) << (8 * (j & 3));
         }
         int4 rec, rec2;
-        rec.x = d | (posn[i] << 8);
+        rec.x = d | (posn[i] << 8) | (size[i] == 1 ? 1 << 16 : 0);         // bit 16: leaf (its u is nobody's ancestor term)
         rec.y = int(w[0]);
         rec.z = int(w[1]);
         rec.w = int(w[2]);
