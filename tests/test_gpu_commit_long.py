@@ -169,3 +169,30 @@ def test_small_batch_takes_single_tiles_and_large_batch_whole_units():
         dp.commit()
         assert dp.status_value() == 0
         assert rel_err(cpu(dp.S), oracle_commit(prob, idx, ln)) <= TOL_FP32
+
+
+def test_commit_with_long_paths_is_cuda_graph_capturable():
+    """Both commit launches go into a captured graph; a replay gives the eager state bit for bit."""
+    prob = synth.make_problem(360, 2, 4, 128, 256, [synth.chain_parent(8) for _ in range(6)])
+    paths = [list(range(n)) for n in (8, 2, 5, 0, 7, 3)]
+    eager = DevProblem(prob)
+    set_paths(eager, prob, paths)
+    eager.commit()
+    assert eager.status_value() == 0
+    dp = DevProblem(prob)
+    set_paths(dp, prob, paths)
+    S0 = dp.S.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        dp.commit()                                        # warm-up outside the capture (first-call device queries)
+        dp.S.copy_(S0)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            dp.commit()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        dp.S.copy_(S0)
+        g.replay()
+        assert dp.status_value() == 0
+        assert torch.equal(dp.S, eager.S)
