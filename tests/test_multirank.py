@@ -111,3 +111,27 @@ def test_launcher_runs_two_ranks_end_to_end_on_cpu():
     assert len(lines) == 1
     line = json.loads(lines[0])
     assert line["impl"] == "reference" and line["n_gpus"] == 2
+
+
+def test_traffic_table_is_read_per_workload_kernel_and_route():
+    """roofline.traffic comes from the table of ncu captures under profiles/: captured bytes x scale, None if absent."""
+    import bench
+    v = bench.ncu_traffic("cfg5", "verify")
+    c = bench.ncu_traffic("cfg5", "commit")
+    assert v is not None and c is not None
+    # one launch streams the 6.4 GB state once (verify) or twice (commit) plus records and outputs
+    assert 8e9 < v < 12e9 and 7e9 < c < 14e9
+    assert bench.ncu_traffic("cfg5-tf32", "verify") is not None
+    assert bench.ncu_traffic("cfg5", "no such kernel") is None and bench.ncu_traffic("nothing", "verify") is None
+
+
+def test_test_only_symbols_are_exported_but_not_declared():
+    """The switches the tests use are reachable through the library, not through the public header."""
+    import ctypes
+    import os
+    from paper_2607_16673_b200 import binding
+    header = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "speca.h")).read()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in ("speca_test_withhold_first_load", "speca_test_commit_long_min_tiles", "speca_test_profiling_build"):
+        assert hasattr(lib, name) and name not in header
+    assert lib.speca_test_profiling_build() == 0, "the committed build configuration carries no profiling counters"
