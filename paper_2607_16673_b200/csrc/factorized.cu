@@ -296,7 +296,7 @@ __device__ __forceinline__ void node_step(float (&ustk)[TP][kMaxDepth], const fl
 // The same step for trees up to MAXD levels deep (the coefficient record is cU[MAXD-1] cV cO[MAXD] cR cG
 // depth-1 offset).  Used for MAXD = 16; the 8-level form above is kept as it is because the shape of its
 // two accumulation chains was tuned.
-template <int TP, int MAXD>
+template <int TP, int MAXD, bool SELF = false>
 __device__ __forceinline__ void node_step_deep(float (&ustk)[TP][MAXD], const float *cf, const float (&Rv)[TP],
                                                const float (&Gv)[TP], const float (&vv)[TP], float (&u_out)[TP],
                                                float (&o_out)[TP], int &off)
@@ -321,7 +321,8 @@ __device__ __forceinline__ void node_step_deep(float (&ustk)[TP][MAXD], const fl
         }
         const float u = u0 + u1;
 #pragma unroll
-        for (int j = 0; j < MAXD; ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        for (int j = 0; j < MAXD - (SELF ? 1 : 0); ++j) ustk[t][j] = (d1 == j) ? u : ustk[t][j];
+        if (SELF) ustk[t][MAXD - 1] = u;
         float o0 = s.y * Gv[t], o1 = 0.f;
 #pragma unroll
         for (int j = 0; j < MAXD; ++j) {
@@ -406,7 +407,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
     const uint32_t tmem_base = *tmem_slot;
 
     constexpr int NS = FUSED ? kStagesFused : kStages;            // ring depth in use
-    constexpr bool kSelfSlot = !DEEP;                             // see node_step
+    constexpr bool kSelfSlot = true;                              // see node_step
     static_assert(DK == 128 || DK == 256, "key width");
     constexpr int NC = DK / kChunkK;                              // K-chunks (state slices) per tile
     constexpr int BROWS = DK == 128 ? kBopRows : kBopRows / 2;    // [K;Q] rows the operand buffers hold
@@ -1100,7 +1101,7 @@ verify_factorized_kernel(const __grid_constant__ CUtensorMap s0_map, const __gri
                     } else {
                         v_[0] = __uint_as_float(uint32_t(vv[i]) << 16);
                     }
-                    if constexpr (DEEP) node_step_deep<TP, MAXD>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
+                    if constexpr (DEEP) node_step_deep<TP, MAXD, kSelfSlot>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
                     else node_step<TP, kSelfSlot>(ustk, coef + (p0 + i) * CS, r_, g_, v_, uo, oo, off);
                     if (p0 + i < n) {
                         if (TP == 2) {
