@@ -196,3 +196,22 @@ def test_commit_with_long_paths_is_cuda_graph_capturable():
         g.replay()
         assert dp.status_value() == 0
         assert torch.equal(dp.S, eager.S)
+
+
+def test_random_batches_of_paths():
+    """Seeded random shapes, trees and accepted paths (every length 0..8 mixed), 12 batches."""
+    rng = np.random.default_rng(370)
+    for it in range(12):
+        d_k = int(rng.choice([64, 128]))
+        d_v = int(rng.choice([64, 128, 256]))
+        B = int(rng.integers(1, 9))
+        parents = deep_parents(B, rng, n_nodes=int(rng.integers(8, 40)))
+        prob = synth.make_problem(371 + it, int(rng.integers(1, 4)), int(rng.integers(1, 5)), d_k, d_v, parents,
+                                  state_std=float(rng.choice([0.02, 0.5])))
+        dp = DevProblem(prob)
+        lengths = [int(rng.integers(0, 9)) for _ in range(B)]
+        idx, ln = set_paths(dp, prob, paths_of_lengths(prob, parents, lengths, rng))
+        dp.commit(check_parent=bool(it & 1))
+        assert dp.status_value() == 0
+        e = rel_err(cpu(dp.S), oracle_commit(prob, idx, ln))
+        assert e <= TOL_FP32, f"batch {it} (d_k={d_k}, d_v={d_v}, lengths {lengths}): state error {e:.3e}"
